@@ -1,0 +1,195 @@
+/*
+ * lagkv.h -- C ABI of the B200 (sm_100a) LagKV KV-cache compression library.
+ *
+ * LagKV (arXiv 2504.04704, Section 2.2) shortens a transformer KV cache without looking
+ * at attention weights.  After an attention-sink prefix of S rows the cache is cut into
+ * partitions of L rows ("lag size").  Partition p is scored against partition p+1: the
+ * per-channel min and max of the next partition (Eq. 7, Eq. 8) normalise the current one
+ * (Eq. 9); the standard deviation over head_dim of every normalised token goes through a
+ * softmax over the partition's tokens (Eq. 10), once for K and once for V, and the two are
+ * added (Eq. 11).  Per head and per partition the k = ceil(r*L) best tokens are kept
+ * (last bullet of Section 2.2); the last full partition plus the Mod(Ls-S, L) trailing
+ * rows stay as a sliding window.  The resulting length is Eq. 12.
+ *
+ * Conventions shared by every entry point
+ *   - All cache pointers are DEVICE pointers to bf16 data, 16-byte aligned; scalars and
+ *     the config struct are host values.  The library allocates no device memory and
+ *     never synchronises the stream, except in lagkv_read_status().
+ *   - A cache is addressed as  base + b*stride_b + h*stride_h + s*stride_s + d  (strides
+ *     in elements, channel stride 1).  A stride given as 0 means "contiguous
+ *     [B, H, S, D]" for the S passed to the call.  Strides must be multiples of 8
+ *     elements (16 bytes).
+ *   - "Layers" have no separate dimension: fold them into B (one allocation
+ *     [layers*B, H, S, D]) so that one call covers a whole model.
+ *   - Every function returning int returns a lagkv_status code (0 = success).
+ *     Errors detected on the host leave all buffers untouched.  Errors detected on the
+ *     device (a bounded wait that ran out, an append that would overflow idx capacity)
+ *     are recorded in the status block at the start of the workspace and reported by
+ *     lagkv_read_status(); the kernels never trap or spin forever.
+ *   - The workspace is caller-owned device memory of at least lagkv_workspace_bytes()
+ *     bytes, 256-byte aligned, cleared once with lagkv_workspace_init() and then reusable
+ *     across calls on the same stream.  Calls sharing a workspace must not overlap.
+ */
+#ifndef LAGKV_H_
+#define LAGKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lagkv_plan_s *lagkv_plan_t;
+
+enum lagkv_status {
+    LAGKV_OK = 0,
+    LAGKV_EINVAL = 1,       /* null pointer, misalignment, bad shape / stride / size  */
+    LAGKV_EUNSUPPORTED = 2, /* valid request this build has no kernel for             */
+    LAGKV_EWORKSPACE = 3,   /* workspace missing or too small                         */
+    LAGKV_ECUDA = 4,        /* CUDA runtime error at launch (left sticky, not cleared)*/
+    LAGKV_ETIMEOUT = 5,     /* device: a bounded wait on an async copy ran out        */
+    LAGKV_ECAPACITY = 6     /* device: append needed more chunks than max_new_chunks  */
+};
+
+enum lagkv_variant {
+    LAGKV_VARIANT_LAGKV = 0,   /* Eq. 7-11: statistics from the next partition        */
+    LAGKV_VARIANT_LOCALKV = 1, /* Eq. 14, Eq. 15: statistics from the partition itself */
+    LAGKV_VARIANT_L2NORM = 2   /* Eq. 16: score = -||K row||_2                        */
+};
+
+typedef struct {
+    int32_t B;          /* sequences (times layers when folded), >= 1                 */
+    int32_t H_kv;       /* KV heads per sequence, >= 1; selection is per KV head      */
+    int32_t D;          /* head_dim; supported: 64, 128, 256 (128 is the tuned case)  */
+    int32_t sink;       /* S: attention-sink rows kept verbatim, >= 0                 */
+    int32_t lag;        /* L: partition size, 2 <= L <= 8192                          */
+    double keep_ratio;  /* r in (0, 1]; k = ceil(r*L - 1e-9) clamped to [1, L]        */
+    int32_t keep_k;     /* if > 0, k directly (overrides keep_ratio)                  */
+    int32_t std_ddof;   /* divisor of the variance is D - std_ddof: 0 or 1            */
+    int32_t variant;    /* enum lagkv_variant                                         */
+    int64_t stride_b;   /* input-cache strides in elements; 0 = contiguous (see top)  */
+    int64_t stride_h;
+    int64_t stride_s;
+    int32_t device;     /* CUDA device ordinal the plan launches on                   */
+} lagkv_config;
+
+/*
+ * Build an immutable plan from a config (Section 2.2: S, L, r fix the whole pass).
+ * Host work plus one-time CUDA attribute queries on cfg->device; no stream work.
+ * On success *out owns host memory freed by lagkv_plan_destroy().
+ */
+int lagkv_plan(const lagkv_config *cfg, lagkv_plan_t *out);
+void lagkv_plan_destroy(lagkv_plan_t plan);
+
+/* k, the rows kept per compressed partition ("only rL tokens will be kept"). */
+int32_t lagkv_keep_count(lagkv_plan_t plan);
+
+/*
+ * Eq. 12 generalised to a cache whose first static_len rows (sink + already compressed
+ * part) are left alone:  static_len + k*(n-1) + L + rem  with n = floor(rest/L),
+ * rem = rest mod L, rest = seq_len - static_len;  seq_len itself when rest < 2L (third
+ * bullet of Section 2.2).  Pure host arithmetic.  static_len < 0 means "the plan's sink".
+ */
+int64_t lagkv_compressed_len(lagkv_plan_t plan, int64_t seq_len, int64_t static_len);
+
+/*
+ * Inverse of Eq. 12 / Eq. 13 as used for the adaptive retention ratio of Section 3.2:
+ * the smallest k in [1, L] whose compression ratio C = 1 - L_R/Ls does not exceed
+ * target_C for a prompt of Ls rows.  Host arithmetic.  Returns k (L when no compression
+ * is possible because Ls < S + 2L).
+ */
+int32_t lagkv_keep_for_target(int64_t Ls, int32_t sink, int32_t lag, double target_C);
+
+/*
+ * Bytes of workspace needed: the status block plus, for lagkv_compress_append(), room
+ * for max_new_chunks*k kept indices per (b, h).  Pass 0 for prefill / gather only.
+ */
+size_t lagkv_workspace_bytes(lagkv_plan_t plan, int32_t max_new_chunks);
+
+/* Clear the status block (async memset on the stream).  Call once per workspace. */
+int lagkv_workspace_init(lagkv_plan_t plan, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream);
+
+/*
+ * One-shot compression of a freshly prefilled cache (first bullet of Section 2.2; Eq. 7-12).
+ * Every sequence has S_in rows.  Out of place; K, V are not modified and may not alias
+ * the outputs.  With L_R = lagkv_compressed_len(plan, S_in, -1):
+ *   K_out, V_out [B, H, L_R, D] bf16 contiguous: sink rows, then for p = 0..n-2 the k kept
+ *                rows of partition p in ascending position, then the window rows.
+ *                Both NULL = indices only.
+ *   idx_out      [B, H, L_R] int32 or NULL: source row of every output row.
+ *   scores_out   [B, H, (n-1)*L] fp32 or NULL: final score (Eq. 11) of every token of a
+ *                compressed partition.
+ * S_in < S + 2L is not an error: the pass is the identity (L_R = S_in).
+ * Asynchronous on cuda_stream (a cudaStream_t, NULL = default stream).
+ */
+int lagkv_compress_prefill(lagkv_plan_t plan, const void *K, const void *V, int64_t S_in,
+                           void *K_out, void *V_out, int32_t *idx_out, float *scores_out,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Incremental (recursive) compression during decode or chunked prefill (Section 2.2,
+ * bullets 2-4; Fig. 1).  In place on caches [B, H, S_cap, D] (the plan's strides, 0 =
+ * contiguous for S_cap).  seq_len[B] and static_len[B] are DEVICE int32 arrays: rows
+ * [0, static_len[b]) are the sink plus everything kept so far, rows up to seq_len[b] are
+ * valid.  For every sequence whose rest = seq_len - static_len is at least 2L the n-1
+ * oldest partitions are scored against their successors, their k kept rows are packed
+ * behind the static part, the window (last full partition + remainder) is moved down
+ * behind them, and the call sets static_len += (n-1)*k, seq_len = static_len + L + rem.
+ * Other sequences are left untouched (decided on the device: no host sync).
+ *   max_new_chunks  capacity: a sequence with n-1 > max_new_chunks is left untouched and
+ *                   LAGKV_ECAPACITY is recorded in the status block.
+ *   idx_out     [B, H, max_new_chunks*k] int32 or NULL: pre-call positions of the rows
+ *               kept by this call (entries of skipped sequences are not written).
+ *   scores_out  [B, H, max_new_chunks*L] fp32 or NULL.
+ * The workspace must have been sized with the same max_new_chunks.
+ */
+int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64_t S_cap,
+                          int32_t *seq_len, int32_t *static_len, int32_t max_new_chunks,
+                          int32_t *idx_out, float *scores_out, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Row gather, the separable part of the compaction (Fig. 1):
+ *   K_out[b,h,j,:] = K[b,h,idx[b,h,j],:],  same for V,  j < n_idx.
+ * K, V use the plan's strides with S_in rows; outputs are contiguous [B, H, n_idx, D].
+ * V / V_out may both be NULL.  idx is a DEVICE int32 array [B, H, n_idx]; every entry
+ * must lie in [0, S_in) -- entries outside are skipped and LAGKV_EINVAL is recorded in
+ * the status block when a workspace is given (workspace may be NULL).
+ */
+int lagkv_gather(lagkv_plan_t plan, const void *K, const void *V, int64_t S_in,
+                 const int32_t *idx, int64_t n_idx, void *K_out, void *V_out, void *workspace,
+                 void *cuda_stream);
+
+/*
+ * Synchronise cuda_stream, copy the status block to the host and clear it.
+ * host_status[0] = first device-side lagkv_status recorded since the last read (0 = none),
+ * host_status[1] = detail (block index), host_status[2] = count of zero-range reference
+ * channels seen, host_status[3] = reserved.  Returns host_status[0], or LAGKV_ECUDA.
+ */
+int lagkv_read_status(lagkv_plan_t plan, void *workspace, void *cuda_stream,
+                      int32_t host_status[4]);
+
+/*
+ * Launch shape the plan uses for a prefill of S_in rows: info[0] = grid, info[1] = block
+ * threads, info[2] = dynamic shared memory bytes, info[3] = kernel launches per call.
+ */
+int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]);
+
+/*
+ * Tuning override: warps per CTA (2, 4 or 8), rows per staged tile (16 or 32), ring
+ * stages per warp (2..8) and resident CTAs per SM to size the grid for (>= 1).  A value
+ * of 0 keeps the planner's choice.  Returns LAGKV_EUNSUPPORTED for a combination that was
+ * not compiled or does not fit shared memory.
+ */
+int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages,
+                    int32_t ctas_per_sm);
+
+const char *lagkv_status_string(int status);
+const char *lagkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAGKV_H_ */

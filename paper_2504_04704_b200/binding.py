@@ -1,0 +1,265 @@
+"""ctypes binding of the C-ABI library declared in ``include/lagkv.h``.
+
+Argument marshalling only: every step of the LagKV compress pass (Section 2.2 of
+arXiv 2504.04704) runs inside the CUDA library.  PyTorch supplies device memory and the
+current stream.  There is no CPU fallback: if ``liblagkv_b200.so`` has not been built
+(``python -c "import __graft_entry__ as g; g.build()"``) the first call raises.
+
+The functions carry the names of the C entry points (``lagkv_plan``,
+``lagkv_compress_prefill``, ``lagkv_compress_append``, ``lagkv_gather`` ...); ``Plan`` is
+a small convenience wrapper that owns the handle and allocates outputs with torch.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+LIB_PATH = Path(__file__).resolve().parent / "liblagkv_b200.so"
+
+LAGKV_OK, LAGKV_EINVAL, LAGKV_EUNSUPPORTED, LAGKV_EWORKSPACE, LAGKV_ECUDA, LAGKV_ETIMEOUT, LAGKV_ECAPACITY = range(7)
+VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
+
+# every symbol include/lagkv.h declares
+EXPORTS = (
+    "lagkv_plan", "lagkv_plan_destroy", "lagkv_keep_count", "lagkv_compressed_len",
+    "lagkv_keep_for_target", "lagkv_workspace_bytes", "lagkv_workspace_init",
+    "lagkv_compress_prefill", "lagkv_compress_append", "lagkv_gather", "lagkv_read_status",
+    "lagkv_launch_info", "lagkv_plan_tune", "lagkv_status_string", "lagkv_version",
+)
+
+
+class LagKVError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class lagkv_config(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("sink", ctypes.c_int32), ("lag", ctypes.c_int32),
+        ("keep_ratio", ctypes.c_double),
+        ("keep_k", ctypes.c_int32), ("std_ddof", ctypes.c_int32), ("variant", ctypes.c_int32),
+        ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_s", ctypes.c_int64),
+        ("device", ctypes.c_int32),
+    ]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Open the CUDA library; a missing build is an error, never a fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build the CUDA library first (__graft_entry__.build()); "
+            "there is no CPU fallback for the LagKV compress pass")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lib.lagkv_plan.restype = ctypes.c_int
+    lib.lagkv_plan.argtypes = [ctypes.POINTER(lagkv_config), ctypes.POINTER(vp)]
+    lib.lagkv_plan_destroy.restype = None
+    lib.lagkv_plan_destroy.argtypes = [vp]
+    lib.lagkv_keep_count.restype = i32
+    lib.lagkv_keep_count.argtypes = [vp]
+    lib.lagkv_compressed_len.restype = i64
+    lib.lagkv_compressed_len.argtypes = [vp, i64, i64]
+    lib.lagkv_keep_for_target.restype = i32
+    lib.lagkv_keep_for_target.argtypes = [i64, i32, i32, ctypes.c_double]
+    lib.lagkv_workspace_bytes.restype = sz
+    lib.lagkv_workspace_bytes.argtypes = [vp, i32]
+    lib.lagkv_workspace_init.restype = ctypes.c_int
+    lib.lagkv_workspace_init.argtypes = [vp, vp, sz, vp]
+    lib.lagkv_compress_prefill.restype = ctypes.c_int
+    lib.lagkv_compress_prefill.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+    lib.lagkv_compress_append.restype = ctypes.c_int
+    lib.lagkv_compress_append.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.lagkv_gather.restype = ctypes.c_int
+    lib.lagkv_gather.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
+    lib.lagkv_read_status.restype = ctypes.c_int
+    lib.lagkv_read_status.argtypes = [vp, vp, vp, ctypes.POINTER(i32 * 4)]
+    lib.lagkv_launch_info.restype = ctypes.c_int
+    lib.lagkv_launch_info.argtypes = [vp, i64, ctypes.POINTER(i32 * 4)]
+    lib.lagkv_plan_tune.restype = ctypes.c_int
+    lib.lagkv_plan_tune.argtypes = [vp, i32, i32, i32, i32]
+    lib.lagkv_status_string.restype = ctypes.c_char_p
+    lib.lagkv_status_string.argtypes = [ctypes.c_int]
+    lib.lagkv_version.restype = ctypes.c_char_p
+    lib.lagkv_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().lagkv_status_string(int(code)).decode()
+
+
+def version() -> str:
+    return load_library().lagkv_version().decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != LAGKV_OK:
+        raise LagKVError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def lagkv_keep_for_target(Ls: int, sink: int, lag: int, target_C: float) -> int:
+    return int(load_library().lagkv_keep_for_target(int(Ls), int(sink), int(lag), float(target_C)))
+
+
+class Plan:
+    """Owns a ``lagkv_plan_t``.  ``device=-1`` makes a host-only plan (integers and launch
+    shapes only; it cannot launch)."""
+
+    def __init__(self, B, H_kv, D, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1,
+                 variant=VARIANT_LAGKV, strides=(0, 0, 0), device=0):
+        lib = load_library()
+        self.cfg = lagkv_config(int(B), int(H_kv), int(D), int(sink), int(lag), float(keep_ratio), int(keep_k),
+                                int(std_ddof), int(variant), int(strides[0]), int(strides[1]), int(strides[2]),
+                                int(device))
+        self.handle = ctypes.c_void_p()
+        _check(lib.lagkv_plan(ctypes.byref(self.cfg), ctypes.byref(self.handle)), "lagkv_plan")
+        self.lib = lib
+        self.device = int(device)
+        self.k = int(lib.lagkv_keep_count(self.handle))
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            self.lib.lagkv_plan_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- host arithmetic
+    def compressed_len(self, seq_len: int, static_len: int = -1) -> int:
+        return int(self.lib.lagkv_compressed_len(self.handle, int(seq_len), int(static_len)))
+
+    def workspace_bytes(self, max_new_chunks: int = 0) -> int:
+        return int(self.lib.lagkv_workspace_bytes(self.handle, int(max_new_chunks)))
+
+    def launch_info(self, S_in: int) -> dict:
+        info = (ctypes.c_int32 * 4)()
+        _check(self.lib.lagkv_launch_info(self.handle, int(S_in), ctypes.byref(info)), "lagkv_launch_info")
+        return {"grid": info[0], "block": info[1], "smem": info[2], "launches": info[3]}
+
+    def tune(self, warps=0, tile_rows=0, stages=0, ctas_per_sm=0) -> None:
+        _check(self.lib.lagkv_plan_tune(self.handle, int(warps), int(tile_rows), int(stages), int(ctas_per_sm)),
+               "lagkv_plan_tune")
+
+    # ---- device work
+    def _dev(self):
+        return torch.device("cuda", self.device)
+
+    def new_workspace(self, max_new_chunks: int = 0) -> torch.Tensor:
+        ws = torch.empty(self.workspace_bytes(max_new_chunks), dtype=torch.uint8, device=self._dev())
+        _check(self.lib.lagkv_workspace_init(self.handle, _ptr(ws), ws.numel(), _stream(self._dev())),
+               "lagkv_workspace_init")
+        return ws
+
+    def read_status(self, workspace: torch.Tensor) -> list[int]:
+        st = (ctypes.c_int32 * 4)()
+        rc = self.lib.lagkv_read_status(self.handle, _ptr(workspace), _stream(self._dev()), ctypes.byref(st))
+        if rc == LAGKV_ECUDA or rc == LAGKV_EINVAL and st[0] != LAGKV_EINVAL:
+            raise LagKVError(rc, "lagkv_read_status")
+        return [int(v) for v in st]
+
+    def _check_cache(self, t: torch.Tensor, name: str):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or t.device.index != self.device:
+            raise TypeError(f"{name} must be a bf16 CUDA tensor on device {self.device}")
+
+    def compress_prefill(self, K, V, workspace, S_in=None, want_rows=True, want_idx=True, want_scores=False,
+                         out=None):
+        """``lagkv_compress_prefill``.  K, V: ``[B, H, S_in, D]`` bf16 (any layout matching the
+        plan's strides).  Returns dict with ``L_R`` and the requested ``K_out``, ``V_out``,
+        ``idx``, ``scores`` tensors.  ``out`` may carry preallocated tensors of the same keys."""
+        self._check_cache(K, "K")
+        self._check_cache(V, "V")
+        c = self.cfg
+        S_in = int(K.shape[2] if S_in is None else S_in)
+        L_R = self.compressed_len(S_in)
+        rest = S_in - c.sink
+        n_c = rest // c.lag - 1 if rest >= 2 * c.lag else 0
+        dev = self._dev()
+        out = dict(out or {})
+        if want_rows:
+            out.setdefault("K_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=torch.bfloat16, device=dev))
+            out.setdefault("V_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=torch.bfloat16, device=dev))
+        if want_idx:
+            out.setdefault("idx", torch.empty((c.B, c.H_kv, L_R), dtype=torch.int32, device=dev))
+        if want_scores:
+            out.setdefault("scores", torch.empty((c.B, c.H_kv, n_c, c.lag), dtype=torch.float32, device=dev))
+        rc = self.lib.lagkv_compress_prefill(
+            self.handle, _ptr(K), _ptr(V), S_in, _ptr(out.get("K_out")), _ptr(out.get("V_out")),
+            _ptr(out.get("idx")), _ptr(out.get("scores")), _ptr(workspace), workspace.numel(), _stream(dev))
+        _check(rc, "lagkv_compress_prefill")
+        out["L_R"], out["n_c"] = L_R, n_c
+        return out
+
+    def compress_append(self, K_cache, V_cache, seq_len, static_len, workspace, max_new_chunks=1,
+                        idx_out=None, scores_out=None):
+        """``lagkv_compress_append``: in place on ``[B, H, S_cap, D]`` caches; ``seq_len`` and
+        ``static_len`` are int32 CUDA tensors ``[B]`` updated by the call."""
+        self._check_cache(K_cache, "K_cache")
+        self._check_cache(V_cache, "V_cache")
+        for t, name in ((seq_len, "seq_len"), (static_len, "static_len")):
+            if t.dtype != torch.int32 or not t.is_cuda or t.numel() != self.cfg.B or not t.is_contiguous():
+                raise TypeError(f"{name} must be a contiguous int32 CUDA tensor [B]")
+        dev = self._dev()
+        rc = self.lib.lagkv_compress_append(
+            self.handle, _ptr(K_cache), _ptr(V_cache), int(K_cache.shape[2]), _ptr(seq_len), _ptr(static_len),
+            int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(workspace), workspace.numel(), _stream(dev))
+        _check(rc, "lagkv_compress_append")
+
+    def gather(self, K, V, idx, workspace=None, S_in=None):
+        """``lagkv_gather``: rows ``idx`` ``[B, H, n_idx]`` int32 of K (and V, may be None)."""
+        self._check_cache(K, "K")
+        c = self.cfg
+        dev = self._dev()
+        if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
+            raise TypeError("idx must be a contiguous int32 CUDA tensor")
+        n_idx = int(idx.shape[-1])
+        S_in = int(K.shape[2] if S_in is None else S_in)
+        K_out = torch.empty((c.B, c.H_kv, n_idx, c.D), dtype=torch.bfloat16, device=dev)
+        V_out = None if V is None else torch.empty_like(K_out)
+        rc = self.lib.lagkv_gather(self.handle, _ptr(K), _ptr(V), S_in, _ptr(idx), n_idx, _ptr(K_out), _ptr(V_out),
+                                   _ptr(workspace), _stream(dev))
+        _check(rc, "lagkv_gather")
+        return K_out, V_out
+
+
+# ---- C-named thin functions ---------------------------------------------------------------
+def lagkv_plan(**kw) -> Plan:
+    return Plan(**kw)
+
+
+def lagkv_plan_destroy(plan: Plan) -> None:
+    plan.close()
+
+
+def lagkv_compress_prefill(plan: Plan, K, V, workspace, **kw):
+    return plan.compress_prefill(K, V, workspace, **kw)
+
+
+def lagkv_compress_append(plan: Plan, K_cache, V_cache, seq_len, static_len, workspace, **kw):
+    return plan.compress_append(K_cache, V_cache, seq_len, static_len, workspace, **kw)
+
+
+def lagkv_gather(plan: Plan, K, V, idx, **kw):
+    return plan.gather(K, V, idx, **kw)

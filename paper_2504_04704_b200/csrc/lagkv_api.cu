@@ -1,0 +1,444 @@
+// LagKV compress pass -- host side of the C ABI declared in include/lagkv.h:
+// argument checks, the planner (integers of Section 2.2 / Eq. 12, launch shapes) and the
+// kernel launches.  No device memory is allocated here.
+#include "lagkv.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "lagkv_kernels.cuh"
+
+using namespace lagkv;
+
+namespace {
+
+typedef void (*stream_kernel_t)(const Params);
+typedef size_t (*smem_fn_t)(int, int);
+
+struct KernelEntry {
+    int D, NW, TR;
+    stream_kernel_t fn;
+    smem_fn_t smem;
+};
+
+#define LAGKV_ENTRY(D, V, NW, TR) \
+    { D, NW, TR, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+
+const KernelEntry kKernels[] = {
+    LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
+    LAGKV_ENTRY(128, 2, 8, 16), LAGKV_ENTRY(128, 2, 4, 16), LAGKV_ENTRY(128, 2, 2, 16),
+    LAGKV_ENTRY(64, 1, 8, 32),  LAGKV_ENTRY(64, 1, 4, 32),  LAGKV_ENTRY(64, 1, 2, 32),
+    LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
+    LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
+    LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+};
+constexpr int kNumKernels = int(sizeof(kKernels) / sizeof(kKernels[0]));
+
+int find_kernel(int D, int NW, int TR) {
+    for (int i = 0; i < kNumKernels; ++i)
+        if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR) return i;
+    return -1;
+}
+
+constexpr int kSmemPerSm = 233472;  // 228 KiB per SM, 1 KiB reserved per resident CTA
+
+}  // namespace
+
+struct lagkv_plan_s {
+    lagkv_config cfg;
+    int k;
+    int sm_count;
+    int max_smem_optin;
+    int kidx;         // index into kKernels
+    int stages;       // ring depth per warp
+    int ctas_per_sm;  // grid sizing for prefill
+    size_t smem;      // dynamic shared memory of the chosen kernel
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (dev >= 0 && cudaGetDevice(&prev) == cudaSuccess && prev != dev)
+            switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+int keep_count(double r, int L) {
+    long long k = (long long)std::ceil(r * (double)L - 1e-9);
+    if (k < 1) k = 1;
+    if (k > L) k = L;
+    return int(k);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Try one launch shape; fills the plan fields on success.
+int apply_shape(lagkv_plan_s* pl, int NW, int TR, int stages, int ctas) {
+    const int kidx = find_kernel(pl->cfg.D, NW, TR);
+    if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
+    const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
+    if (smem > size_t(pl->max_smem_optin)) return LAGKV_EUNSUPPORTED;
+    if ((smem + 1024) * size_t(ctas) > size_t(kSmemPerSm)) return LAGKV_EUNSUPPORTED;
+    if (pl->cfg.device >= 0 &&
+        cudaFuncSetAttribute(reinterpret_cast<const void*>(kKernels[kidx].fn),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+        return LAGKV_ECUDA;
+    pl->kidx = kidx;
+    pl->stages = stages;
+    pl->ctas_per_sm = ctas;
+    pl->smem = smem;
+    return LAGKV_OK;
+}
+
+// Planner default: more warps and deeper rings for long partitions, many small CTAs for
+// short ones (the per-partition select phase is a fixed cost that other CTAs must hide).
+int choose_shape(lagkv_plan_s* pl) {
+    const int L = pl->cfg.lag;
+    struct Cand { int NW, TR, stages, ctas; };
+    Cand cands[8];
+    int nc = 0;
+    if (L >= 1024) {
+        cands[nc++] = {8, 32, 3, 1};
+        cands[nc++] = {8, 32, 2, 1};
+    }
+    if (L >= 256) {
+        cands[nc++] = {4, 32, 3, 2};
+        cands[nc++] = {4, 32, 2, 2};
+    }
+    cands[nc++] = {2, 16, 4, 6};
+    cands[nc++] = {2, 16, 3, 4};
+    cands[nc++] = {2, 16, 2, 2};
+    cands[nc++] = {2, 16, 2, 1};
+    int rc = LAGKV_EUNSUPPORTED;
+    for (int i = 0; i < nc; ++i) {
+        rc = apply_shape(pl, cands[i].NW, cands[i].TR, cands[i].stages, cands[i].ctas);
+        if (rc == LAGKV_OK || rc == LAGKV_ECUDA) return rc;
+    }
+    return rc;
+}
+
+struct Strides {
+    long long sb, sh, ss;
+};
+int resolve_strides(const lagkv_config& c, int64_t S, Strides* out) {
+    long long ss = c.stride_s ? c.stride_s : c.D;
+    long long sh = c.stride_h ? c.stride_h : (long long)S * ss;
+    long long sb = c.stride_b ? c.stride_b : (long long)c.H_kv * sh;
+    if (ss < c.D || (ss % 8) || (sh % 8) || (sb % 8) || sh < 0 || sb < 0) return LAGKV_EINVAL;
+    out->sb = sb;
+    out->sh = sh;
+    out->ss = ss;
+    return LAGKV_OK;
+}
+
+int check_launch() {
+    return cudaPeekAtLastError() == cudaSuccess ? LAGKV_OK : LAGKV_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
+    if (cfg == nullptr || out == nullptr) return LAGKV_EINVAL;
+    *out = nullptr;
+    if (cfg->B < 1 || cfg->H_kv < 1 || cfg->sink < 0 || cfg->lag < 2 || cfg->lag > 8192) return LAGKV_EINVAL;
+    if (cfg->std_ddof != 0 && cfg->std_ddof != 1) return LAGKV_EINVAL;
+    if (cfg->keep_k < 0 || cfg->keep_k > cfg->lag) return LAGKV_EINVAL;
+    if (cfg->keep_k == 0 && !(cfg->keep_ratio > 0.0 && cfg->keep_ratio <= 1.0)) return LAGKV_EINVAL;
+    if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
+    if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
+    if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
+    if (cfg->variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
+    if (cfg->D != 64 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
+    if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
+
+    lagkv_plan_s* pl = new (std::nothrow) lagkv_plan_s();
+    if (pl == nullptr) return LAGKV_EINVAL;
+    pl->cfg = *cfg;
+    pl->k = cfg->keep_k > 0 ? cfg->keep_k : keep_count(cfg->keep_ratio, cfg->lag);
+    DeviceGuard guard(cfg->device);
+    if (cfg->device < 0) {  // host-only plan: nominal B200 figures, launches are refused
+        pl->sm_count = 148;
+        pl->max_smem_optin = 232448;
+    } else if (cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess ||
+               cudaDeviceGetAttribute(&pl->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device) !=
+                   cudaSuccess) {
+        delete pl;
+        return LAGKV_ECUDA;
+    }
+    const int rc = choose_shape(pl);
+    if (rc != LAGKV_OK) {
+        delete pl;
+        return rc;
+    }
+    *out = pl;
+    return LAGKV_OK;
+}
+
+void lagkv_plan_destroy(lagkv_plan_t plan) { delete plan; }
+
+int32_t lagkv_keep_count(lagkv_plan_t plan) { return plan ? plan->k : 0; }
+
+int64_t lagkv_compressed_len(lagkv_plan_t plan, int64_t seq_len, int64_t static_len) {
+    if (plan == nullptr) return -1;
+    const int64_t L = plan->cfg.lag, st = static_len < 0 ? plan->cfg.sink : static_len;
+    const int64_t rest = seq_len - st;
+    if (rest < 2 * L) return seq_len;
+    return st + int64_t(plan->k) * (rest / L - 1) + L + rest % L;
+}
+
+int32_t lagkv_keep_for_target(int64_t Ls, int32_t sink, int32_t lag, double target_C) {
+    if (lag < 1 || Ls < sink + 2ll * lag) return lag;
+    const int64_t n = (Ls - sink) / lag, rem = (Ls - sink) % lag;
+    for (int32_t k = 1; k <= lag; ++k) {
+        const int64_t L_R = sink + int64_t(k) * (n - 1) + lag + rem;
+        const double C = 1.0 - double(L_R) / double(Ls);
+        if (C <= target_C + 1e-12) return k;
+    }
+    return lag;
+}
+
+size_t lagkv_workspace_bytes(lagkv_plan_t plan, int32_t max_new_chunks) {
+    if (plan == nullptr || max_new_chunks < 0) return 0;
+    size_t bytes = kStatusWords * sizeof(int32_t);
+    bytes += size_t(plan->cfg.B) * plan->cfg.H_kv * size_t(max_new_chunks) * plan->k * sizeof(int32_t);
+    return (bytes + 255) & ~size_t(255);
+}
+
+int lagkv_workspace_init(lagkv_plan_t plan, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (plan == nullptr || plan->cfg.device < 0) return LAGKV_EINVAL;
+    if (workspace == nullptr || workspace_bytes < kStatusWords * sizeof(int32_t)) return LAGKV_EWORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
+    DeviceGuard guard(plan->cfg.device);
+    if (cudaMemsetAsync(workspace, 0, kStatusWords * sizeof(int32_t), static_cast<cudaStream_t>(cuda_stream)) !=
+        cudaSuccess)
+        return LAGKV_ECUDA;
+    return LAGKV_OK;
+}
+
+int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, void* K_out,
+                           void* V_out, int32_t* idx_out, float* scores_out, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    if (plan == nullptr || K == nullptr || V == nullptr || plan->cfg.device < 0) return LAGKV_EINVAL;
+    if ((K_out == nullptr) != (V_out == nullptr)) return LAGKV_EINVAL;
+    if (S_in < 0 || S_in > 0x7fffffffll - 65536) return LAGKV_EINVAL;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out)) return LAGKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(idx_out) & 3u) || (reinterpret_cast<uintptr_t>(scores_out) & 3u))
+        return LAGKV_EINVAL;
+    if (K_out != nullptr && (K_out == K || V_out == V || K_out == V || V_out == K)) return LAGKV_EINVAL;
+    if (workspace == nullptr || workspace_bytes < kStatusWords * sizeof(int32_t)) return LAGKV_EWORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
+    const lagkv_config& c = plan->cfg;
+    Strides st;
+    if (resolve_strides(c, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    if (S_in == 0) return LAGKV_OK;
+
+    DeviceGuard guard(c.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const long long U = (long long)c.B * c.H_kv;
+    const int64_t rest = S_in - c.sink;
+
+    if (rest < 2ll * c.lag) {  // pass skipped: identity
+        if (K_out == nullptr && idx_out == nullptr) return LAGKV_OK;
+        const long long total = U * S_in * (c.D / 8);
+        const int block = 256;
+        const long long want = (total + block - 1) / block;
+        const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
+        lagkv_copy_kernel<<<grid, block, 0, stream>>>(
+            static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), st.sb, st.sh, st.ss, c.H_kv,
+            int(S_in), c.D / 8, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), idx_out, U);
+        return check_launch();
+    }
+
+    Params P;
+    std::memset(&P, 0, sizeof P);
+    P.K = static_cast<const uint16_t*>(K);
+    P.V = static_cast<const uint16_t*>(V);
+    P.K_out = static_cast<uint16_t*>(K_out);
+    P.V_out = static_cast<uint16_t*>(V_out);
+    P.idx_out = idx_out;
+    P.scores_out = scores_out;
+    P.status = static_cast<int32_t*>(workspace);
+    P.sb = st.sb;
+    P.sh = st.sh;
+    P.ss = st.ss;
+    P.B = c.B;
+    P.H = c.H_kv;
+    P.L = c.lag;
+    P.k = plan->k;
+    P.ddof = c.std_ddof;
+    P.variant = c.variant;
+    P.mode = MODE_PREFILL;
+    P.S_in = int(S_in);
+    P.sink = c.sink;
+    P.n = int(rest / c.lag);
+    P.rem = int(rest % c.lag);
+    P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
+    P.total_slots = U * P.n;
+    P.stages = plan->stages;
+
+    const KernelEntry& ke = kKernels[plan->kidx];
+    long long grid = (long long)plan->sm_count * plan->ctas_per_sm;
+    if (grid > P.total_slots) grid = P.total_slots;
+    void* args[] = {&P};
+    if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)grid), dim3(ke.NW * 32), args,
+                         plan->smem, stream) != cudaSuccess)
+        return LAGKV_ECUDA;
+    return check_launch();
+}
+
+int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
+                          int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (plan == nullptr || K_cache == nullptr || V_cache == nullptr || seq_len == nullptr || static_len == nullptr ||
+        plan->cfg.device < 0)
+        return LAGKV_EINVAL;
+    if (S_cap < 1 || S_cap > 0x7fffffffll - 65536 || max_new_chunks < 1) return LAGKV_EINVAL;
+    if (!aligned16(K_cache) || !aligned16(V_cache) || K_cache == V_cache) return LAGKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(idx_out) & 3u) || (reinterpret_cast<uintptr_t>(scores_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(seq_len) & 3u) || (reinterpret_cast<uintptr_t>(static_len) & 3u))
+        return LAGKV_EINVAL;
+    if (workspace == nullptr) return LAGKV_EWORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
+    const size_t need = idx_out ? kStatusWords * sizeof(int32_t) : lagkv_workspace_bytes(plan, max_new_chunks);
+    if (workspace_bytes < need) return LAGKV_EWORKSPACE;
+    const lagkv_config& c = plan->cfg;
+    Strides st;
+    if (resolve_strides(c, S_cap, &st) != LAGKV_OK) return LAGKV_EINVAL;
+
+    DeviceGuard guard(c.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    Params P;
+    std::memset(&P, 0, sizeof P);
+    P.K = static_cast<const uint16_t*>(K_cache);
+    P.V = static_cast<const uint16_t*>(V_cache);
+    P.K_out = static_cast<uint16_t*>(K_cache);
+    P.V_out = static_cast<uint16_t*>(V_cache);
+    P.scores_out = scores_out;
+    P.seq_len = seq_len;
+    P.static_len = static_len;
+    P.status = static_cast<int32_t*>(workspace);
+    P.kept_pos = idx_out ? idx_out : static_cast<int32_t*>(workspace) + kStatusWords;
+    P.sb = st.sb;
+    P.sh = st.sh;
+    P.ss = st.ss;
+    P.B = c.B;
+    P.H = c.H_kv;
+    P.L = c.lag;
+    P.k = plan->k;
+    P.ddof = c.std_ddof;
+    P.variant = c.variant;
+    P.mode = MODE_APPEND;
+    P.S_in = int(S_cap);
+    P.sink = c.sink;
+    P.max_chunks = max_new_chunks;
+    P.stages = plan->stages;
+
+    const KernelEntry& ke = kKernels[plan->kidx];
+    const long long U = (long long)c.B * c.H_kv;
+    void* args[] = {&P};
+    if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)U), dim3(ke.NW * 32), args,
+                         plan->smem, stream) != cudaSuccess)
+        return LAGKV_ECUDA;
+    lagkv_update_lengths_kernel<<<(c.B + 127) / 128, 128, 0, stream>>>(seq_len, static_len, c.B, c.lag, plan->k,
+                                                                       max_new_chunks, int(S_cap));
+    return check_launch();
+}
+
+int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, const int32_t* idx, int64_t n_idx,
+                 void* K_out, void* V_out, void* workspace, void* cuda_stream) {
+    if (plan == nullptr || K == nullptr || K_out == nullptr || idx == nullptr || plan->cfg.device < 0)
+        return LAGKV_EINVAL;
+    if ((V == nullptr) != (V_out == nullptr)) return LAGKV_EINVAL;
+    if (S_in < 1 || S_in > 0x7fffffffll - 65536 || n_idx < 0) return LAGKV_EINVAL;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out)) return LAGKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return LAGKV_EINVAL;
+    const lagkv_config& c = plan->cfg;
+    Strides st;
+    if (resolve_strides(c, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    if (n_idx == 0) return LAGKV_OK;
+    DeviceGuard guard(c.device);
+    const long long U = (long long)c.B * c.H_kv;
+    const long long total = U * n_idx * (c.D / 8);
+    const int block = 256;
+    const long long want = (total + block - 1) / block;
+    const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
+    lagkv_gather_kernel<<<grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), st.sb, st.sh, st.ss, c.H_kv, int(S_in),
+        c.D / 8, idx, n_idx, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), U,
+        static_cast<int32_t*>(workspace));
+    return check_launch();
+}
+
+int lagkv_read_status(lagkv_plan_t plan, void* workspace, void* cuda_stream, int32_t host_status[4]) {
+    if (plan == nullptr || workspace == nullptr || host_status == nullptr || plan->cfg.device < 0)
+        return LAGKV_EINVAL;
+    DeviceGuard guard(plan->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(host_status, workspace, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return LAGKV_ECUDA;
+    if (cudaMemsetAsync(workspace, 0, kStatusWords * sizeof(int32_t), stream) != cudaSuccess) return LAGKV_ECUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return LAGKV_ECUDA;
+    return host_status[0];
+}
+
+int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
+    if (plan == nullptr || info == nullptr || S_in < 0) return LAGKV_EINVAL;
+    const lagkv_config& c = plan->cfg;
+    const long long U = (long long)c.B * c.H_kv;
+    const int64_t rest = S_in - c.sink;
+    if (rest < 2ll * c.lag) {
+        const long long total = U * S_in * (c.D / 8);
+        const long long want = (total + 255) / 256;
+        info[0] = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
+        info[1] = 256;
+        info[2] = 0;
+        info[3] = S_in > 0 ? 1 : 0;
+        return LAGKV_OK;
+    }
+    long long grid = (long long)plan->sm_count * plan->ctas_per_sm;
+    const long long slots = U * (rest / c.lag);
+    info[0] = int(grid < slots ? grid : slots);
+    info[1] = kKernels[plan->kidx].NW * 32;
+    info[2] = int(plan->smem);
+    info[3] = 1;
+    return LAGKV_OK;
+}
+
+int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages, int32_t ctas_per_sm) {
+    if (plan == nullptr) return LAGKV_EINVAL;
+    DeviceGuard guard(plan->cfg.device);
+    const KernelEntry& cur = kKernels[plan->kidx];
+    lagkv_plan_s trial = *plan;
+    const int rc = apply_shape(&trial, warps ? warps : cur.NW, tile_rows ? tile_rows : cur.TR,
+                               stages ? stages : plan->stages, ctas_per_sm ? ctas_per_sm : plan->ctas_per_sm);
+    if (rc == LAGKV_OK) *plan = trial;
+    return rc;
+}
+
+const char* lagkv_status_string(int status) {
+    switch (status) {
+        case LAGKV_OK: return "ok";
+        case LAGKV_EINVAL: return "invalid argument";
+        case LAGKV_EUNSUPPORTED: return "unsupported configuration";
+        case LAGKV_EWORKSPACE: return "workspace missing or too small";
+        case LAGKV_ECUDA: return "CUDA error";
+        case LAGKV_ETIMEOUT: return "device wait timed out";
+        case LAGKV_ECAPACITY: return "append needs more chunks than max_new_chunks";
+        default: return "unknown status";
+    }
+}
+
+const char* lagkv_version(void) { return "lagkv-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,865 @@
+// LagKV compress pass -- sm_100a device code.
+//
+// One kernel family does the whole pass of Section 2.2 (arXiv 2504.04704) with a single
+// read of the cache from HBM:
+//
+//   * Work is a list of "slots" (unit u = (b, h), partition p), ordered so that inside a
+//     unit the partitions come in DESCENDING p.  A CTA walks a contiguous range of that
+//     list.  When it streams partition p it already holds the per-channel min/max of
+//     partition p+1 (Eq. 7, Eq. 8) from the previous step, so in one pass over the rows it
+//     (a) normalises and accumulates the per-token sum and sum of squares over head_dim
+//     (Eq. 9, Eq. 10) and (b) collects p's own min/max for use by p-1.
+//   * Each warp owns a private ring of shared-memory tiles filled by bulk async copies
+//     (cp.async.bulk + mbarrier complete_tx); lane 0 of the warp is its own producer, so
+//     the streaming loop has no block-level synchronisation.  Even warps stream K, odd
+//     warps stream V.
+//   * At the end of a partition the CTA runs softmax over the L tokens for K and V, adds
+//     them (Eq. 11), selects the k best with a radix select on the fp32 bit pattern
+//     (ties to the lower index) and copies the kept rows straight to the output layout
+//     (rows come back from L2, which they passed through moments before).
+//
+// No tensor cores: the pass is a streaming reduction / selection / gather.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lagkv {
+
+constexpr int kStatusWords = 64;  // 256-byte status block at the start of the workspace
+constexpr int kMaxWarps = 8;
+
+enum { MODE_PREFILL = 0, MODE_APPEND = 1 };
+enum { ST_OK = 0, ST_EINVAL = 1, ST_ETIMEOUT = 5, ST_ECAPACITY = 6 };
+
+struct Params {
+    const uint16_t* K;  // input cache (prefill) / cache updated in place (append)
+    const uint16_t* V;
+    uint16_t* K_out;  // prefill: contiguous [U, L_R, D]; append: same memory as K / V
+    uint16_t* V_out;
+    int32_t* idx_out;
+    float* scores_out;
+    const int32_t* seq_len;     // append: device [B]
+    const int32_t* static_len;  // append: device [B]
+    int32_t* kept_pos;          // append: [U, max_chunks * k] pre-call positions of kept rows
+    int32_t* status;            // status block
+    long long sb, sh, ss;       // cache strides in elements
+    long long total_slots;      // prefill: U * n
+    int B, H, L, k, ddof, variant, mode;
+    int S_in, sink, n, rem, L_R;  // prefill
+    int max_chunks;               // append
+    int stages;                   // ring depth per warp
+};
+
+// ------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+// packed pair of fp32 in one 64-bit register (Blackwell f32x2 arithmetic)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// two bf16 in one word -> two fp32 (exact)
+__device__ __forceinline__ f32x2 bf2_to_f32x2(uint32_t w) {
+    return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ uint4 ld_nc(const uint4* p) { return __ldg(p); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ void record_status(int32_t* status, int code, int detail) {
+    if (status != nullptr && atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+// order-preserving map fp32 -> uint32 (larger float <=> larger key)
+__device__ __forceinline__ uint32_t float_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ------------------------------------------------------------------------- geometry / smem
+template <int D_, int V_, int NW_, int TR_>
+struct Geo {
+    static constexpr int D = D_;           // head_dim
+    static constexpr int V = V_;           // 16-byte vectors per thread per row
+    static constexpr int NW = NW_;         // warps per CTA (even: K warps, odd: V warps)
+    static constexpr int TR = TR_;         // rows per staged tile
+    static constexpr int NT = NW * 32;
+    static constexpr int WT = NW / 2;      // warps per tensor
+    static constexpr int VPR = D / 8;      // 16-byte vectors per row
+    static constexpr int LPR = VPR / V;    // lanes per row
+    static constexpr int RPL = 32 / LPR;   // rows per warp-wide load
+    static constexpr int NV = TR / RPL;    // row partials per thread per tile
+    static constexpr int NWORD = 4 * V;    // packed bf16x2 words per thread per row
+    static constexpr int TILE_BYTES = TR * D * 2;
+    static_assert(LPR * V == VPR && RPL * LPR == 32 && NV * RPL == TR, "bad geometry");
+    static_assert(NV >= 1 && NV <= LPR, "tile too tall for the transposed reduction");
+    static_assert(NW >= 2 && NW <= kMaxWarps && (NW % 2) == 0, "bad warp count");
+};
+
+struct SelScratch {
+    float red[4][kMaxWarps];
+    int hist[256];
+    int wsum[kMaxWarps];
+    int bin;
+    int krem;
+};
+
+template <class G>
+__host__ __device__ constexpr size_t smem_ring_bytes(int stages) {
+    return size_t(G::NW) * stages * G::TILE_BYTES;
+}
+template <class G>
+__host__ __device__ inline size_t smem_total_bytes(int stages, int L) {
+    size_t s = smem_ring_bytes<G>(stages);         // tile rings
+    s += size_t(G::NW) * stages * 8;               // mbarriers
+    s += size_t(2) * G::WT * 2 * (G::D / 2) * 4;   // per-warp min/max partials
+    s += sizeof(SelScratch);
+    s = (s + 15) & ~size_t(15);
+    s += size_t(2) * ((L + 3) & ~3) * 4;           // sigma / score / kept arrays
+    return s + 128;                                // alignment slack
+}
+
+// -------------------------------------------------------------- cross-lane row reduction
+// v[i] holds this lane's partial for row-slot i; LPR consecutive lanes share the rows.
+// After the call lane cg holds the full sum of slot (cg >> log2(LPR/NV)) in v[0].
+template <int NV, int LPR>
+__device__ __forceinline__ void transposed_reduce(float (&v)[NV], int cg) {
+    int o = LPR / 2;
+#pragma unroll
+    for (int n = NV; n > 1; n >>= 1, o >>= 1) {
+        const bool up = (cg & o) != 0;
+        const int h = n / 2;
+#pragma unroll
+        for (int i = 0; i < h; ++i) {
+            const float send = up ? v[i] : v[i + h];
+            const float keep = up ? v[i + h] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+#pragma unroll
+    for (; o >= 1; o >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+}
+
+// ---------------------------------------------------------------------------- tile math
+// One staged tile of one tensor: rows [0, nrows) valid.  Updates the packed per-channel
+// min / max; when SCORE, also writes sigma (Std. of Eq. 10) for every valid row.
+template <class G, bool SCORE, bool FULL>
+__device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int nrows,
+                                             const f32x2 (&a2)[G::NWORD], const f32x2 (&b2)[G::NWORD],
+                                             uint32_t (&mn)[G::NWORD], uint32_t (&mx)[G::NWORD],
+                                             float* __restrict__ sig_out, float inv_D, float inv_Dm,
+                                             int lane) {
+    const int cg = lane % G::LPR, rl = lane / G::LPR;
+    float p1[G::NV], p2[G::NV];
+#pragma unroll
+    for (int i = 0; i < G::NV; ++i) {
+        const int row = i * G::RPL + rl;
+        const bool valid = FULL || row < nrows;
+        f32x2 s1 = 0ull, s2 = 0ull;
+#pragma unroll
+        for (int v = 0; v < G::V; ++v) {
+            const uint4 q = tile[row * G::VPR + v * G::LPR + cg];
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int j = v * 4 + c;
+                if (valid) {
+                    mn[j] = bf2_min(mn[j], w[c]);
+                    mx[j] = bf2_max(mx[j], w[c]);
+                }
+                if (SCORE) {
+                    const f32x2 y = fma2(bf2_to_f32x2(w[c]), a2[j], b2[j]);  // Eq. 9 (centred)
+                    s1 = add2(s1, y);
+                    s2 = fma2(y, y, s2);
+                }
+            }
+        }
+        if (SCORE) {
+            float lo, hi;
+            unpack2(s1, lo, hi);
+            p1[i] = lo + hi;
+            unpack2(s2, lo, hi);
+            p2[i] = lo + hi;
+        }
+    }
+    if (SCORE) {
+        transposed_reduce<G::NV, G::LPR>(p1, cg);
+        transposed_reduce<G::NV, G::LPR>(p2, cg);
+        constexpr int DUP = G::LPR / G::NV;
+        const int row = (cg / DUP) * G::RPL + rl;
+        if ((cg % DUP) == 0 && (FULL || row < nrows)) {
+            const float mean = p1[0] * inv_D;
+            float var = (p2[0] - p1[0] * mean) * inv_Dm;
+            var = fmaxf(var, 0.0f);
+            sig_out[row] = sqrtf(var);
+        }
+    }
+}
+
+// -------------------------------------------------------------- softmax + top-k (block)
+// In: sg0 = sigma(K), sg1 = sigma(V), L entries each (shared memory).
+// Out: sg0 = final score (Eq. 11); kept = (int*)sg1 holds the k selected indices ascending.
+// All NT threads of the CTA must call; contains block barriers.
+template <int NT>
+__device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool single_tensor,
+                                 float* __restrict__ scores_g, SelScratch& sc, int tid) {
+    constexpr int NWARP = NT / 32;
+    const int lane = tid & 31, warp = tid >> 5;
+
+    if (!single_tensor) {
+        // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
+        float m0 = -INFINITY, m1 = -INFINITY;
+        for (int t = tid; t < L; t += NT) {
+            m0 = fmaxf(m0, sg0[t]);
+            m1 = fmaxf(m1, sg1[t]);
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+            m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+        }
+        if (lane == 0) {
+            sc.red[0][warp] = m0;
+            sc.red[1][warp] = m1;
+        }
+        __syncthreads();
+        m0 = sc.red[0][0];
+        m1 = sc.red[1][0];
+#pragma unroll
+        for (int w = 1; w < NWARP; ++w) {
+            m0 = fmaxf(m0, sc.red[0][w]);
+            m1 = fmaxf(m1, sc.red[1][w]);
+        }
+        float s0 = 0.f, s1 = 0.f;
+        for (int t = tid; t < L; t += NT) {
+            const float e0 = expf(sg0[t] - m0), e1 = expf(sg1[t] - m1);
+            sg0[t] = e0;
+            sg1[t] = e1;
+            s0 += e0;
+            s1 += e1;
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        }
+        if (lane == 0) {
+            sc.red[2][warp] = s0;
+            sc.red[3][warp] = s1;
+        }
+        __syncthreads();
+        s0 = sc.red[2][0];
+        s1 = sc.red[3][0];
+#pragma unroll
+        for (int w = 1; w < NWARP; ++w) {
+            s0 += sc.red[2][w];
+            s1 += sc.red[3][w];
+        }
+        // ---- Eq. 11
+        for (int t = tid; t < L; t += NT) {
+            const float s = sg0[t] / s0 + sg1[t] / s1;
+            sg0[t] = s;
+            if (scores_g != nullptr) scores_g[t] = s;
+        }
+    } else if (scores_g != nullptr) {
+        for (int t = tid; t < L; t += NT) scores_g[t] = sg0[t];
+    }
+    __syncthreads();
+
+    // ---- radix select: key of the k-th largest score, 8 bits per pass
+    uint32_t prefix = 0, mask = 0;
+    int krem = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += NT) sc.hist[i] = 0;
+        __syncthreads();
+        for (int t0 = 0; t0 < L; t0 += NT) {
+            const int t = t0 + tid;
+            const bool in = t < L;
+            const uint32_t key = in ? float_key(sg0[t]) : 0u;
+            const bool act = in && ((key & mask) == prefix);
+            const int bin = act ? int((key >> shift) & 255u) : -1 - lane;
+            // warp-aggregated histogram update
+            const uint32_t peers = __match_any_sync(0xffffffffu, bin);
+            if (act && lane == (__ffs(peers) - 1)) atomicAdd(&sc.hist[bin], __popc(peers));
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane owns bins [8*lane, 8*lane+8); walk from the top bin down
+            int c[8], tot = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                c[i] = sc.hist[lane * 8 + i];
+                tot += c[i];
+            }
+            int above = tot;  // inclusive suffix sum over lanes >= this one
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_down_sync(0xffffffffu, above, o);
+                if (lane + o < 32) above += v;
+            }
+            const int excl = above - tot;  // count in bins of higher lanes
+            if (excl < krem && krem <= above) {
+                int acc = excl;
+#pragma unroll
+                for (int i = 7; i >= 0; --i) {
+                    if (acc < krem && krem <= acc + c[i]) {
+                        sc.bin = lane * 8 + i;
+                        sc.krem = krem - acc;
+                    }
+                    acc += c[i];
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= uint32_t(sc.bin) << shift;
+        mask |= 255u << shift;
+        krem = sc.krem;
+    }
+    // prefix = key of the k-th largest; krem = how many tokens with exactly that key are kept
+
+    // ---- positions: each thread owns a contiguous index range, block scan over counts
+    const int E = (L + NT - 1) / NT;
+    const int t_lo = min(tid * E, L), t_hi = min(t_lo + E, L);
+    int cgt = 0, ceq = 0;
+    for (int t = t_lo; t < t_hi; ++t) {
+        const uint32_t key = float_key(sg0[t]);
+        cgt += key > prefix;
+        ceq += key == prefix;
+    }
+    int packed = cgt | (ceq << 16), incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) sc.wsum[warp] = incl;
+    __syncthreads();  // also: every thread is done reading sg1, so kept[] may overwrite it
+    int off = 0;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w)
+        if (w < warp) off += sc.wsum[w];
+    const int excl = off + incl - packed;
+    int pgt = excl & 0xffff, peq = excl >> 16;
+    int* kept = reinterpret_cast<int*>(sg1);
+    for (int t = t_lo; t < t_hi; ++t) {
+        const uint32_t key = float_key(sg0[t]);
+        if (key > prefix) {
+            kept[pgt + min(peq, krem)] = t;
+            ++pgt;
+        } else if (key == prefix) {
+            if (peq < krem) kept[pgt + peq] = t;
+            ++peq;
+        }
+    }
+    __syncthreads();
+}
+
+// --------------------------------------------------------------------------- row copies
+// dst rows [dst_row0, +nrows) <- src rows [src_row0, +nrows), both tensors, disjoint buffers.
+template <int NT, int VPR>
+__device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
+                          long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
+                          int src_row0, int dst_row0, int nrows, int32_t* __restrict__ idx_dst, int tid) {
+    if (dstK != nullptr) {
+        const long long items = (long long)nrows * 2 * VPR;
+        constexpr int U = 4;
+        for (long long base = 0; base < items; base += NT * U) {
+            uint4 buf[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const long long i = base + u * NT + tid;
+                if (i < items) {
+                    const int vec = int(i % VPR);
+                    const long long r2 = i / VPR;
+                    const int row = int(r2 >> 1);
+                    const uint16_t* s = (r2 & 1) ? srcV : srcK;
+                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + (src_row0 + row) * ss) + vec);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const long long i = base + u * NT + tid;
+                if (i < items) {
+                    const int vec = int(i % VPR);
+                    const long long r2 = i / VPR;
+                    const int row = int(r2 >> 1);
+                    uint16_t* d = (r2 & 1) ? dstV : dstK;
+                    st_stream(reinterpret_cast<uint4*>(d + (long long)(dst_row0 + row) * (VPR * 8)) + vec, buf[u]);
+                }
+            }
+        }
+    }
+    if (idx_dst != nullptr)
+        for (int r = tid; r < nrows; r += NT) idx_dst[dst_row0 + r] = src_row0 + r;
+}
+
+// kept rows of one partition -> output (prefill, out of place)
+template <int NT, int VPR>
+__device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
+                          long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
+                          int src_row0, int dst_row0, const int* __restrict__ kept, int k,
+                          int32_t* __restrict__ idx_dst, int tid) {
+    if (dstK != nullptr) {
+        const int items = k * 2 * VPR;
+        constexpr int U = 4;
+        for (int base = 0; base < items; base += NT * U) {
+            uint4 buf[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i = base + u * NT + tid;
+                if (i < items) {
+                    const int vec = i % VPR, r2 = i / VPR, j = r2 >> 1;
+                    const uint16_t* s = (r2 & 1) ? srcV : srcK;
+                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + (long long)(src_row0 + kept[j]) * ss) + vec);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i = base + u * NT + tid;
+                if (i < items) {
+                    const int vec = i % VPR, r2 = i / VPR, j = r2 >> 1;
+                    uint16_t* d = (r2 & 1) ? dstV : dstK;
+                    st_stream(reinterpret_cast<uint4*>(d + (long long)(dst_row0 + j) * (VPR * 8)) + vec, buf[u]);
+                }
+            }
+        }
+    }
+    if (idx_dst != nullptr)
+        for (int j = tid; j < k; j += NT) idx_dst[dst_row0 + j] = src_row0 + kept[j];
+}
+
+// In-place move inside one cache (append): dst row = dst_row0 + j, src row = src_of(j),
+// dst <= src for every j and both ascending.  Every batch is loaded into registers by the
+// whole CTA, then a barrier, then stored, so no row is overwritten before it is read.
+template <int NT, int VPR, class SrcOf>
+__device__ void move_rows_inplace(uint16_t* K, uint16_t* V, long long ss, int dst_row0, int nrows,
+                                  SrcOf src_of, int tid) {
+    const long long items = (long long)nrows * 2 * VPR;
+    constexpr int U = 4;
+    for (long long base = 0; base < items; base += NT * U) {
+        uint4 buf[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long i = base + u * NT + tid;
+            if (i < items) {
+                const int vec = int(i % VPR);
+                const long long r2 = i / VPR;
+                const int j = int(r2 >> 1);
+                const uint16_t* s = (r2 & 1) ? V : K;
+                buf[u] = *(reinterpret_cast<const uint4*>(s + (long long)src_of(j) * ss) + vec);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long i = base + u * NT + tid;
+            if (i < items) {
+                const int vec = int(i % VPR);
+                const long long r2 = i / VPR;
+                const int j = int(r2 >> 1);
+                uint16_t* d = (r2 & 1) ? V : K;
+                *(reinterpret_cast<uint4*>(d + (long long)(dst_row0 + j) * ss) + vec) = buf[u];
+            }
+        }
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------- kernel
+template <class G>
+__global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int NS = P.stages;
+    unsigned char* ring = sm;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ring + smem_ring_bytes<G>(NS));
+    uint32_t* stats = reinterpret_cast<uint32_t*>(bars + G::NW * NS);  // [2][WT][2][D/2]
+    SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * G::WT * 2 * (G::D / 2));
+    float* sg = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
+    const int Lp = (P.L + 3) & ~3;
+    float* sg0 = sg;
+    float* sg1 = sg + Lp;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tensor = warp & 1, wj = warp >> 1;
+    const int cg = lane % G::LPR, rl = lane / G::LPR;
+    const int L = P.L, k = P.k;
+    const int ntiles = (L + G::TR - 1) / G::TR;
+    const bool contiguous = (P.ss == G::D);
+
+    // ---- which slots does this CTA walk?
+    long long s_first, s_hi;  // owned slots [s_first, s_hi)
+    int n, stat_rows, unit_fixed = 0, rem = 0;
+    if (P.mode == MODE_PREFILL) {
+        n = P.n;
+        stat_rows = P.sink;
+        s_first = P.total_slots * blockIdx.x / gridDim.x;
+        s_hi = P.total_slots * (blockIdx.x + 1) / gridDim.x;
+    } else {
+        unit_fixed = blockIdx.x;
+        const int b = unit_fixed / P.H;
+        const int seq = P.seq_len[b];
+        stat_rows = P.static_len[b];
+        const int rest = seq - stat_rows;
+        if (seq > P.S_in || stat_rows < 0 || rest < 0) {  // lengths that do not describe this cache
+            if (tid == 0) record_status(P.status, ST_EINVAL, b);
+            return;
+        }
+        if (rest < 2 * L) return;  // third bullet of Section 2.2: skip
+        n = rest / L;
+        rem = rest % L;
+        if (n - 1 > P.max_chunks) {
+            if (tid == 0) record_status(P.status, ST_ECAPACITY, b);
+            return;
+        }
+        s_first = 0;
+        s_hi = n;
+    }
+    if (s_first >= s_hi) return;
+    // a range that starts in the middle of a unit first re-reads the partition above it
+    const bool extra = (P.mode == MODE_PREFILL) && (s_first % n) != 0;
+    const long long s_lo = extra ? s_first - 1 : s_first;
+
+    auto slot_unit = [&](long long s) -> int { return P.mode == MODE_PREFILL ? int(s / n) : unit_fixed; };
+    auto slot_part = [&](long long s) -> int { return n - 1 - int(s % n); };
+    const uint16_t* tbase = tensor ? P.V : P.K;
+    auto unit_base = [&](const uint16_t* base, int u) -> const uint16_t* {
+        return base + (long long)(u / P.H) * P.sb + (long long)(u % P.H) * P.sh;
+    };
+
+    // ---- per-warp ring
+    const uint32_t ring_w = smem_u32(ring) + uint32_t(warp) * NS * G::TILE_BYTES;
+    const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
+    if (lane == 0)
+        for (int i = 0; i < NS; ++i) mbar_init(bar_w + 8 * i, 1);
+    fence_mbar_init();
+    fence_proxy_async();
+    __syncthreads();
+
+    const bool has_tiles = wj < ntiles;
+    long long ps = s_lo;  // producer cursor: next tile to request
+    int pt = wj;
+    int pslot = 0;
+    auto issue_next = [&]() {  // warp-collective
+        if (!has_tiles || ps >= s_hi) return;
+        const int u = slot_unit(ps), p = slot_part(ps);
+        const int row0 = stat_rows + p * L + pt * G::TR;
+        const int rows = min(G::TR, L - pt * G::TR);
+        const uint16_t* src = unit_base(tbase, u) + (long long)row0 * P.ss;
+        const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
+        const uint32_t bar = bar_w + 8 * pslot;
+        const uint32_t bytes = uint32_t(rows) * G::D * 2;
+        if (lane == 0) {
+            fence_proxy_async();
+            mbar_arrive_expect_tx(bar, bytes);
+        }
+        if (contiguous) {
+            if (lane == 0) bulk_g2s(dst, src, bytes, bar);
+        } else {
+            __syncwarp();
+            for (int r = lane; r < rows; r += 32)
+                bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+        }
+        pt += G::WT;
+        if (pt >= ntiles) {
+            pt = wj;
+            ++ps;
+        }
+        if (++pslot == NS) pslot = 0;
+    };
+    for (int i = 0; i < NS; ++i) issue_next();
+
+    int cslot = 0;
+    uint32_t cparity = 0;
+    bool timed_out = false;
+    const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
+
+    f32x2 a2[G::NWORD], b2[G::NWORD];
+#pragma unroll
+    for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
+    bool have_ref = false;
+
+    for (long long s = s_lo; s < s_hi; ++s) {
+        const int u = slot_unit(s), p = slot_part(s);
+        const bool top = (p == n - 1);
+        const bool score = !top && s >= s_first && have_ref;
+
+        uint32_t mn[G::NWORD], mx[G::NWORD];
+#pragma unroll
+        for (int j = 0; j < G::NWORD; ++j) {
+            mn[j] = 0x7f807f80u;  // +inf, +inf
+            mx[j] = 0xff80ff80u;  // -inf, -inf
+        }
+        float* sig = tensor ? sg1 : sg0;
+
+        for (int t = wj; t < ntiles; t += G::WT) {
+            const uint32_t bar = bar_w + 8 * cslot;
+            if (!mbar_try_wait(bar, cparity)) {
+                const unsigned long long t0 = global_timer_ns();
+                bool ok = false;
+                for (int it = 0; it < (1 << 26) && !ok; ++it) {
+                    ok = mbar_try_wait(bar, cparity);
+                    if (!ok && (it & 255) == 255 && global_timer_ns() - t0 > 1000000000ull) break;
+                }
+                if (!ok) {
+                    timed_out = true;
+                    if (lane == 0) record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+                }
+            }
+            const uint4* tile = reinterpret_cast<const uint4*>(ring + size_t(warp) * NS * G::TILE_BYTES +
+                                                               size_t(cslot) * G::TILE_BYTES);
+            const int nrows = min(G::TR, L - t * G::TR);
+            float* so = sig + t * G::TR;
+            if (nrows == G::TR) {
+                if (score) process_tile<G, true, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                else process_tile<G, false, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+            } else {
+                if (score) process_tile<G, true, false>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                else process_tile<G, false, false>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+            }
+            __syncwarp();
+            issue_next();  // refill the slot just drained
+            if (++cslot == NS) {
+                cslot = 0;
+                cparity ^= 1u;
+            }
+        }
+
+        // ---- this partition's min / max (Eq. 7, Eq. 8): lanes sharing channels, then warps
+#pragma unroll
+        for (int j = 0; j < G::NWORD; ++j) {
+#pragma unroll
+            for (int o = G::LPR; o < 32; o <<= 1) {
+                mn[j] = bf2_min(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
+                mx[j] = bf2_max(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+            }
+        }
+        if (rl == 0) {
+            uint32_t* st = stats + ((tensor * G::WT + wj) * 2) * (G::D / 2);
+#pragma unroll
+            for (int v = 0; v < G::V; ++v)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    st[(v * G::LPR + cg) * 4 + c] = mn[v * 4 + c];
+                    st[(G::D / 2) + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
+                }
+        }
+        __syncthreads();
+
+        // ---- select and emit partition p
+        if (score) {
+            const int n_c = n - 1;
+            float* scores_g = nullptr;
+            if (P.scores_out != nullptr)
+                scores_g = (P.mode == MODE_PREFILL)
+                               ? P.scores_out + ((long long)u * n_c + p) * L
+                               : P.scores_out + ((long long)u * P.max_chunks + p) * L;
+            score_and_select<G::NT>(sg0, sg1, L, k, false, scores_g, sc, tid);
+            const int* kept = reinterpret_cast<const int*>(sg1);
+            if (P.mode == MODE_PREFILL) {
+                emit_kept<G::NT, G::VPR>(unit_base(P.K, u), unit_base(P.V, u), P.ss,
+                                         P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr,
+                                         P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr,
+                                         stat_rows + p * L, stat_rows + p * k, kept, k,
+                                         P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr, tid);
+            } else {
+                int32_t* kp = P.kept_pos + ((long long)u * P.max_chunks + p) * k;
+                for (int j = tid; j < k; j += G::NT) kp[j] = stat_rows + p * L + kept[j];
+            }
+        }
+
+        // ---- coefficients for the next (lower) partition from this one's statistics:
+        //      y = (z - mid) / range, a shift of Eq. 9 by -1/2 that leaves the std unchanged
+        {
+            uint32_t fmn[G::NWORD], fmx[G::NWORD];
+#pragma unroll
+            for (int j = 0; j < G::NWORD; ++j) {
+                fmn[j] = 0x7f807f80u;
+                fmx[j] = 0xff80ff80u;
+            }
+            for (int w = 0; w < G::WT; ++w) {
+                const uint32_t* st = stats + ((tensor * G::WT + w) * 2) * (G::D / 2);
+#pragma unroll
+                for (int v = 0; v < G::V; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        fmn[v * 4 + c] = bf2_min(fmn[v * 4 + c], st[(v * G::LPR + cg) * 4 + c]);
+                        fmx[v * 4 + c] = bf2_max(fmx[v * 4 + c], st[(G::D / 2) + (v * G::LPR + cg) * 4 + c]);
+                    }
+            }
+            int zero_range = 0;
+#pragma unroll
+            for (int j = 0; j < G::NWORD; ++j) {
+                const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
+                const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
+                const float r0 = hi0 - lo0, r1 = hi1 - lo1;
+                const float a0 = r0 > 0.f ? 1.0f / r0 : 0.f, a1 = r1 > 0.f ? 1.0f / r1 : 0.f;
+                const float c0 = r0 > 0.f ? -(0.5f * (lo0 + hi0)) * a0 : -0.5f;
+                const float c1 = r1 > 0.f ? -(0.5f * (lo1 + hi1)) * a1 : -0.5f;
+                zero_range += !(r0 > 0.f);
+                zero_range += !(r1 > 0.f);
+                a2[j] = pack2(a0, a1);
+                b2[j] = pack2(c0, c1);
+            }
+            if (zero_range != 0 && wj == 0 && rl == 0 && P.status != nullptr) atomicAdd(P.status + 2, zero_range);
+            have_ref = true;
+        }
+
+        // ---- rows copied verbatim (prefill): window with the top slot, sink with slot p = 0
+        if (P.mode == MODE_PREFILL && s >= s_first) {
+            const uint16_t* uk = unit_base(P.K, u);
+            const uint16_t* uv = unit_base(P.V, u);
+            uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
+            uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
+            int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
+            if (top)
+                copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, stat_rows + (n - 1) * L, stat_rows + (n - 1) * k,
+                                         L + P.rem, oi, tid);
+            if (p == 0) copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, 0, 0, stat_rows, oi, tid);
+        }
+        if (p == 0) have_ref = false;  // next slot belongs to another unit
+        __syncthreads();
+    }
+
+    // ---- append: pack kept rows behind the static part, then slide the window down
+    if (P.mode == MODE_APPEND) {
+        const int u = unit_fixed;
+        uint16_t* ck = const_cast<uint16_t*>(unit_base(P.K, u));
+        uint16_t* cv = const_cast<uint16_t*>(unit_base(P.V, u));
+        const int n_c = n - 1;
+        const int32_t* kp = P.kept_pos + (long long)u * P.max_chunks * k;
+        if (k < L) {
+            move_rows_inplace<G::NT, G::VPR>(ck, cv, P.ss, stat_rows, n_c * k,
+                                             [&](int j) { return kp[j]; }, tid);
+            const int src0 = stat_rows + n_c * L;
+            move_rows_inplace<G::NT, G::VPR>(ck, cv, P.ss, stat_rows + n_c * k, L + rem,
+                                             [&](int j) { return src0 + j; }, tid);
+        }
+    }
+
+    // a wait that ran out may have left copies in flight: give them one more bounded chance
+    if (timed_out) {
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
+    }
+}
+
+// append: lengths after the pass (run as a second launch so that every CTA of the main
+// kernel has read the old values)
+__global__ void lagkv_update_lengths_kernel(int32_t* seq_len, int32_t* static_len, int B, int L, int k,
+                                            int max_chunks, int S_cap) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int seq = seq_len[b], st = static_len[b];
+    const int rest = seq - st;
+    if (rest < 2 * L || st < 0 || seq > S_cap) return;
+    const int n = rest / L, rem = rest % L;
+    if (n - 1 > max_chunks) return;
+    const int ns = st + (n - 1) * k;
+    static_len[b] = ns;
+    seq_len[b] = ns + L + rem;
+}
+
+// identity pass (S_in < S + 2L) and plain strided -> contiguous copy
+__global__ void lagkv_copy_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V, long long sb,
+                                  long long sh, long long ss, int H, int rows, int vpr, uint16_t* __restrict__ K_out,
+                                  uint16_t* __restrict__ V_out, int32_t* __restrict__ idx_out, long long units) {
+    const long long per_unit = (long long)rows * vpr;
+    const long long total = units * per_unit;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long u = i / per_unit, r = (i % per_unit) / vpr;
+        const int vec = int(i % vpr);
+        const long long src = (u / H) * sb + (u % H) * sh + r * ss;
+        if (K_out) reinterpret_cast<uint4*>(K_out + (u * rows + r) * vpr * 8)[vec] = __ldg(reinterpret_cast<const uint4*>(K + src) + vec);
+        if (V_out) reinterpret_cast<uint4*>(V_out + (u * rows + r) * vpr * 8)[vec] = __ldg(reinterpret_cast<const uint4*>(V + src) + vec);
+        if (idx_out && vec == 0) idx_out[u * rows + r] = int(r);
+    }
+}
+
+// gather: out[u, j, :] = in[u, idx[u, j], :]
+__global__ void lagkv_gather_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V, long long sb,
+                                    long long sh, long long ss, int H, int S_in, int vpr,
+                                    const int32_t* __restrict__ idx, long long n_idx, uint16_t* __restrict__ K_out,
+                                    uint16_t* __restrict__ V_out, long long units, int32_t* status) {
+    const long long per_unit = n_idx * vpr;
+    const long long total = units * per_unit;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long u = i / per_unit, j = (i % per_unit) / vpr;
+        const int vec = int(i % vpr);
+        const int r = idx[u * n_idx + j];
+        if (r < 0 || r >= S_in) {
+            if (vec == 0) record_status(status, ST_EINVAL, int(u));
+            continue;
+        }
+        const long long src = (u / H) * sb + (u % H) * sh + (long long)r * ss;
+        reinterpret_cast<uint4*>(K_out + (u * n_idx + j) * vpr * 8)[vec] = __ldg(reinterpret_cast<const uint4*>(K + src) + vec);
+        if (V_out) reinterpret_cast<uint4*>(V_out + (u * n_idx + j) * vpr * 8)[vec] = __ldg(reinterpret_cast<const uint4*>(V + src) + vec);
+    }
+}
+
+}  // namespace lagkv

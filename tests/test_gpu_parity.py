@@ -1,0 +1,367 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle
+on the same seeded bf16 inputs.
+
+Bars (see also the design document):
+  * per-token scores within 1e-4 absolute of the oracle (binding) and, tighter, within
+    SCORE_REL_TOL of the mean score 2/L;
+  * kept index sets identical to the oracle's, except partitions where the oracle's own
+    k-th / (k+1)-th score gap is below the tolerance (counted, and additionally required
+    to be explained by the measured score error: every token in the symmetric difference
+    lies within 2*eps_p of the oracle's k-th score);
+  * the GPU's selection is exactly the top-k (ties to the lower index) of the GPU's own
+    fp32 scores -- bit-exact, no tolerance;
+  * compacted K/V rows bit-exact given the indices; sink and window bit-identical.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_04704_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+SCORE_ABS_TOL = 1e-4     # binding tolerance on scores
+SCORE_REL_TOL = 2e-5     # tight: |gpu - oracle| <= SCORE_REL_TOL * (2 / L)
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2504_04704_b200 import binding as b
+    b.load_library()
+    return b
+
+
+def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None):
+    """Compare a GPU prefill result ``out`` (numpy arrays) with the oracle on bit patterns."""
+    ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof)
+    B, H, S, D = Kb.shape
+    assert out["L_R"] == ref["L_R"]
+    n_c = ref["n_c"]
+    idx = out["idx"]
+    # rows bit-exact given the GPU's own indices
+    take = idx[..., None].astype(np.int64)
+    np.testing.assert_array_equal(out["K_out"], np.take_along_axis(Kb, take, axis=2))
+    np.testing.assert_array_equal(out["V_out"], np.take_along_axis(Vb, take, axis=2))
+    if n_c == 0:
+        np.testing.assert_array_equal(idx, ref["idx"])
+        return {"mismatch_partitions": 0, "max_abs": 0.0, "max_rel": 0.0}
+    # sink and window
+    np.testing.assert_array_equal(idx[..., :sink], ref["idx"][..., :sink])
+    np.testing.assert_array_equal(idx[..., sink + n_c * k:], ref["idx"][..., sink + n_c * k:])
+    # scores
+    gs = out["scores"].astype(np.float64)
+    err = np.abs(gs - ref["scores"])
+    max_abs = float(err.max())
+    max_rel = float(err.max() * L / 2.0)
+    assert max_abs <= SCORE_ABS_TOL, f"score error {max_abs}"
+    assert max_rel <= SCORE_REL_TOL, f"score error relative to 2/L: {max_rel}"
+    # the GPU's selection is the exact top-k of its own fp32 scores
+    s32 = out["scores"]
+    order = np.argsort(-s32, axis=-1, kind="stable")[..., :k]
+    own = np.sort(order, axis=-1) + (sink + np.arange(n_c) * L)[None, None, :, None]
+    got = idx[..., sink:sink + n_c * k].reshape(B, H, n_c, k)
+    np.testing.assert_array_equal(got, own)
+    # index sets against the oracle
+    want = ref["idx"][..., sink:sink + n_c * k].reshape(B, H, n_c, k)
+    bad = np.argwhere((got != want).any(-1))
+    loose_unexplained = tight_unexplained = 0
+    for b, h, p in bad:
+        sc = ref["scores"][b, h, p]
+        srt = np.sort(sc)[::-1]
+        gap = srt[k - 1] - srt[k] if k < L else np.inf
+        if gap >= SCORE_ABS_TOL:
+            loose_unexplained += 1
+        eps = err[b, h, p].max()
+        diff = np.setxor1d(got[b, h, p], want[b, h, p]) - (sink + p * L)
+        if np.any(np.abs(sc[diff] - srt[k - 1]) > 2 * eps):
+            tight_unexplained += 1
+    assert loose_unexplained == 0
+    assert tight_unexplained == 0
+    res = {"mismatch_partitions": int(len(bad)), "partitions": int(B * H * n_c), "max_abs": max_abs, "max_rel": max_rel}
+    if stats is not None:
+        stats.update(res)
+    return res
+
+
+def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=None, sigma_k=1.0, layout="bhsd"):
+    K, V = synth.make_kv(B, H, S, D, seed=seed, sigma_k=sigma_k, device="cuda:0")
+    strides = (0, 0, 0)
+    Kd, Vd = K, V
+    if layout == "bshd":        # cache stored [B, S, H, D]; passed as a strided [B, H, S, D] view
+        Kd = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        Vd = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        strides = (S * H * D, D, H * D)
+    elif layout == "padded":    # rows padded to D + 8 elements
+        Kp = torch.zeros((B, H, S, D + 8), dtype=torch.bfloat16, device="cuda:0")
+        Vp = torch.zeros_like(Kp)
+        Kp[..., :D], Vp[..., :D] = K, V
+        Kd, Vd = Kp, Vp
+        strides = (H * S * (D + 8), S * (D + 8), D + 8)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, std_ddof=ddof, strides=strides, device=0)
+    if tune:
+        plan.tune(**tune)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill(Kd, Vd, ws, S_in=S, want_scores=True)
+    st = plan.read_status(ws)
+    assert st[0] == 0, f"device status {st}"
+    host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
+            "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
+    return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host)
+
+
+# ------------------------------------------------------------------------------- prefill
+def test_config0_tiny_prefill(binding, oracle):
+    """B=1, H=8, D=128, S=4096, sink=16, L=128, r=0.25, seed 0."""
+    res = run_prefill(binding, oracle, 1, 8, 128, 4096, 16, 128, 32, seed=0)
+    assert res["partitions"] == 8 * 30
+
+
+@pytest.mark.parametrize("L,k,S_extra", [(64, 4, 60), (100, 25, 7), (72, 72, 0), (256, 1, 255), (512, 128, 3),
+                                         (1024, 256, 1008), (2048, 256, 100), (37, 5, 36), (2, 1, 1)])
+def test_prefill_lag_sweep(binding, oracle, L, k, S_extra):
+    """Partition sizes across several tiles with ragged last tiles and remainders."""
+    n = 5 if L >= 512 else 9
+    run_prefill(binding, oracle, 2, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L)
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_prefill_head_dims(binding, oracle, D, ddof):
+    run_prefill(binding, oracle, 1, 4, D, 16 + 6 * 128 + 37, 16, 128, 32, seed=D + ddof, ddof=ddof)
+
+
+@pytest.mark.parametrize("layout", ["bshd", "padded"])
+def test_prefill_strided_layouts(binding, oracle, layout):
+    run_prefill(binding, oracle, 2, 4, 128, 8 + 4 * 96 + 11, 8, 96, 24, seed=3, layout=layout)
+
+
+@pytest.mark.parametrize("warps,tile_rows,stages", [(8, 32, 3), (8, 32, 2), (4, 32, 4), (2, 32, 3), (8, 16, 4),
+                                                    (4, 16, 2), (2, 16, 8)])
+def test_prefill_every_launch_shape(binding, oracle, warps, tile_rows, stages):
+    run_prefill(binding, oracle, 1, 6, 128, 16 + 7 * 320 + 100, 16, 320, 80, seed=warps * 100 + tile_rows + stages,
+                tune=dict(warps=warps, tile_rows=tile_rows, stages=stages, ctas_per_sm=1))
+
+
+def test_prefill_many_units_ranges_start_mid_unit(binding, oracle):
+    """More (b, h) units than CTAs and a partition count that does not divide evenly, so
+    CTA ranges begin inside units and re-read a reference partition."""
+    run_prefill(binding, oracle, 7, 5, 128, 3 + 6 * 64 + 5, 3, 64, 16, seed=77,
+                tune=dict(warps=2, tile_rows=16, stages=3, ctas_per_sm=1))
+
+
+def test_prefill_heavy_outliers(binding, oracle):
+    run_prefill(binding, oracle, 1, 8, 128, 16 + 8 * 256 + 200, 16, 256, 32, seed=5, sigma_k=1.5)
+
+
+def test_prefill_sink_zero_and_minimal(binding, oracle):
+    run_prefill(binding, oracle, 1, 2, 128, 2 * 128, 0, 128, 32, seed=9)       # n = 2, no sink, no remainder
+
+
+def test_prefill_identity_when_too_short(binding, oracle):
+    run_prefill(binding, oracle, 2, 2, 128, 16 + 2 * 128 - 1, 16, 128, 32, seed=11)
+
+
+def test_constant_partition_ties_keep_first_k(binding, oracle):
+    """All tokens of a partition identical: every score equals 2/L and the tie rule keeps
+    the first k rows (exact, no tolerance)."""
+    B, H, D, sink, L, k = 1, 2, 128, 4, 64, 16
+    S = sink + 3 * L
+    K, V = synth.make_kv(B, H, S, D, seed=13, device="cuda:0")
+    K[:, :, sink:sink + L] = K[:, :, sink:sink + 1]
+    V[:, :, sink:sink + L] = V[:, :, sink:sink + 1]
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill(K, V, ws, want_scores=True)
+    assert plan.read_status(ws)[0] == 0
+    idx = out["idx"].cpu().numpy()
+    assert np.all(idx[..., sink:sink + k] == sink + np.arange(k))
+    ref = oracle.compress(synth.to_bits(K), synth.to_bits(V), sink, L, k)
+    np.testing.assert_array_equal(idx[..., :sink + k], ref["idx"][..., :sink + k])
+
+
+def test_zero_range_channel(binding, oracle):
+    """A reference channel that is constant over the lag partition contributes y = 0."""
+    B, H, D, sink, L, k = 1, 2, 128, 4, 64, 16
+    S = sink + 3 * L + 5
+    K, V = synth.make_kv(B, H, S, D, seed=15, device="cuda:0")
+    K[:, :, sink + L:sink + 2 * L, 7] = 1.5
+    V[:, :, sink + L:sink + 2 * L, 100] = -0.25
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill(K, V, ws, want_scores=True)
+    st = plan.read_status(ws)
+    assert st[0] == 0 and st[2] >= 4      # two heads x (one K + one V channel)
+    host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
+            "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
+    check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host)
+
+
+def test_indices_only_and_rows_only(binding, oracle):
+    B, H, D, sink, L, k = 1, 3, 128, 8, 128, 32
+    S = sink + 4 * L + 17
+    K, V = synth.make_kv(B, H, S, D, seed=17, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace()
+    full = plan.compress_prefill(K, V, ws)
+    only_idx = plan.compress_prefill(K, V, ws, want_rows=False)
+    only_rows = plan.compress_prefill(K, V, ws, want_idx=False)
+    assert torch.equal(full["idx"], only_idx["idx"])
+    assert torch.equal(full["K_out"], only_rows["K_out"]) and torch.equal(full["V_out"], only_rows["V_out"])
+    assert plan.read_status(ws)[0] == 0
+
+
+def test_power_of_two_channel_rescale_is_bit_invariant(binding):
+    """z -> 2^e_c z on every row (exact in bf16) leaves the normalised values, hence the fp32
+    scores and the selection, bit-identical."""
+    B, H, D, sink, L, k = 1, 4, 128, 0, 128, 32
+    S = 5 * L
+    K, V = synth.make_kv(B, H, S, D, seed=19, device="cuda:0")
+    g = torch.Generator(device="cuda:0").manual_seed(1)
+    e = torch.randint(-5, 6, (1, H, 1, D), generator=g, device="cuda:0").float()
+    K2, V2 = (K.float() * torch.exp2(e)).to(torch.bfloat16), (V.float() * torch.exp2(-e)).to(torch.bfloat16)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace()
+    a = plan.compress_prefill(K, V, ws, want_scores=True)
+    b = plan.compress_prefill(K2, V2, ws, want_scores=True)
+    assert torch.equal(a["idx"], b["idx"])
+    assert torch.equal(a["scores"], b["scores"])
+
+
+# -------------------------------------------------------------------------------- gather
+def test_gather(binding, oracle):
+    B, H, D, S = 2, 3, 128, 500
+    K, V = synth.make_kv(B, H, S, D, seed=21, device="cuda:0")
+    g = torch.Generator(device="cuda:0").manual_seed(2)
+    idx = torch.randint(0, S, (B, H, 77), generator=g, device="cuda:0", dtype=torch.int32)
+    plan = binding.Plan(B, H, D, 4, 64, keep_k=16, device=0)
+    ws = plan.new_workspace()
+    Ko, Vo = plan.gather(K, V, idx, workspace=ws)
+    np.testing.assert_array_equal(synth.to_bits(Ko), oracle.gather(synth.to_bits(K), idx.cpu().numpy()))
+    np.testing.assert_array_equal(synth.to_bits(Vo), oracle.gather(synth.to_bits(V), idx.cpu().numpy()))
+    assert plan.read_status(ws)[0] == 0
+    Ko2, none = plan.gather(K, None, idx)
+    assert none is None and torch.equal(Ko, Ko2)
+    # an index outside [0, S) is skipped and reported, not dereferenced
+    idx[0, 0, 3] = S
+    plan.gather(K, V, idx, workspace=ws)
+    assert plan.read_status(ws)[0] == binding.LAGKV_EINVAL
+
+
+# -------------------------------------------------------------------------------- append
+def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chunks, seed, tune=None, give_idx=True):
+    K, V = synth.make_kv(B, H, S_cap, D, seed=seed, device="cuda:0")
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
+    stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    if tune:
+        plan.tune(**tune)
+    ws = plan.new_workspace(max_chunks)
+    idx_out = torch.full((B, H, max_chunks * k), -1, dtype=torch.int32, device="cuda:0") if give_idx else None
+    plan.compress_append(K, V, seq_d, stat_d, ws, max_new_chunks=max_chunks, idx_out=idx_out)
+    st = plan.read_status(ws)
+    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k)
+    return dict(K=synth.to_bits(K), V=synth.to_bits(V), seq=seq_d.cpu().numpy(), stat=stat_d.cpu().numpy(),
+                idx=None if idx_out is None else idx_out.cpu().numpy(), status=st,
+                Kr=Kr, Vr=Vr, seq_r=seq_r, stat_r=stat_r, kept=kept, K0=Kb, V0=Vb)
+
+
+def check_append(r, B):
+    assert r["status"][0] == 0, r["status"]
+    np.testing.assert_array_equal(r["seq"], r["seq_r"])
+    np.testing.assert_array_equal(r["stat"], r["stat_r"])
+    for b in range(B):
+        n = int(r["seq_r"][b])
+        np.testing.assert_array_equal(r["K"][b, :, :n], r["Kr"][b, :, :n])
+        np.testing.assert_array_equal(r["V"][b, :, :n], r["Vr"][b, :, :n])
+        if r["idx"] is not None and r["kept"][b].shape[1]:
+            m = r["kept"][b].shape[1]
+            np.testing.assert_array_equal(r["idx"][b, :, :m], r["kept"][b])
+
+
+def test_append_single_chunk_ragged_batch(binding, oracle):
+    """Decode-style trigger: some sequences just reached 2L of new rows, others not yet."""
+    sink, L, k = 16, 128, 32
+    stat = [16, 16 + 3 * k, 16, 16 + 7 * k]
+    seq = [stat[0] + 2 * L, stat[1] + 2 * L + 5, stat[2] + 2 * L - 1, stat[3] + L]
+    r = append_case(binding, oracle, 4, 3, 128, 1200, sink, L, k, seq, stat, 1, seed=31)
+    check_append(r, 4)
+    # skipped sequences are bit-identical everywhere
+    np.testing.assert_array_equal(r["K"][2], r["K0"][2])
+    np.testing.assert_array_equal(r["V"][3], r["V0"][3])
+    # rows at and beyond the pre-call seq_len are never written
+    for b in range(4):
+        np.testing.assert_array_equal(r["K"][b, :, seq[b]:], r["K0"][b, :, seq[b]:])
+
+
+@pytest.mark.parametrize("L,k,chunks", [(64, 16, 4), (96, 96, 2), (256, 1, 3), (512, 128, 2)])
+def test_append_multi_chunk(binding, oracle, L, k, chunks):
+    sink = 8
+    stat = [sink, sink + 2 * k]
+    seq = [stat[0] + (chunks + 1) * L + 3, stat[1] + (chunks + 1) * L + L - 1]
+    r = append_case(binding, oracle, 2, 2, 128, seq[1] + 9, sink, L, k, seq, stat, chunks, seed=L + k,
+                    give_idx=(L != 96))
+    check_append(r, 2)
+
+
+def test_append_capacity_error_leaves_sequence_alone(binding, oracle):
+    sink, L, k = 4, 64, 16
+    stat, seq = [4, 4], [4 + 2 * L, 4 + 4 * L]      # second sequence needs 3 chunks
+    r = append_case(binding, oracle, 2, 2, 128, 300, sink, L, k, seq, stat, 1, seed=41)
+    assert r["status"][0] == binding.LAGKV_ECAPACITY and r["status"][1] == 1
+    np.testing.assert_array_equal(r["K"][1], r["K0"][1])
+    assert r["seq"][1] == seq[1] and r["stat"][1] == stat[1]
+    assert r["seq"][0] == r["seq_r"][0]
+    np.testing.assert_array_equal(r["K"][0, :, :r["seq"][0]], r["Kr"][0, :, :r["seq"][0]])
+
+
+def test_prefill_equals_incremental_on_gpu(binding, oracle):
+    """One-shot prefill == prefill of S+2L rows followed by token-by-token appends with an
+    append call after every token (most calls skip on the device)."""
+    B, H, D, sink, L, k = 2, 2, 128, 4, 32, 8
+    total = sink + 2 * L + 3 * L + 11
+    K, V = synth.make_kv(B, H, total, D, seed=51, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace(1)
+    one = plan.compress_prefill(K, V, ws)
+    Kc = torch.zeros((B, H, total, D), dtype=torch.bfloat16, device="cuda:0")
+    Vc = torch.zeros_like(Kc)
+    first = sink + 2 * L
+    Kc[:, :, :first], Vc[:, :, :first] = K[:, :, :first], V[:, :, :first]
+    seq = torch.full((B,), first, dtype=torch.int32, device="cuda:0")
+    stat = torch.full((B,), sink, dtype=torch.int32, device="cuda:0")
+    plan.compress_append(Kc, Vc, seq, stat, ws, max_new_chunks=1)
+    for t in range(first, total):
+        s = int(seq[0])
+        Kc[:, :, s], Vc[:, :, s] = K[:, :, t], V[:, :, t]
+        seq += 1
+        plan.compress_append(Kc, Vc, seq, stat, ws, max_new_chunks=1)
+    assert plan.read_status(ws)[0] == 0
+    assert seq.tolist() == [one["L_R"]] * B
+    assert stat.tolist() == [sink + 4 * k] * B
+    assert torch.equal(Kc[:, :, :one["L_R"]], one["K_out"])
+    assert torch.equal(Vc[:, :, :one["L_R"]], one["V_out"])
+
+
+# ----------------------------------------------------------------------- argument checks
+def test_argument_errors(binding):
+    with pytest.raises(binding.LagKVError) as e:
+        binding.Plan(1, 1, 100, 4, 64, device=0)
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+    with pytest.raises(binding.LagKVError) as e:
+        binding.Plan(1, 1, 128, 4, 1, device=0)
+    assert e.value.code == binding.LAGKV_EINVAL
+    plan = binding.Plan(1, 2, 128, 4, 64, keep_k=16, device=0)
+    K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
+    small = torch.empty(16, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(binding.LagKVError) as e:
+        plan.compress_prefill(K, V, small)
+    assert e.value.code == binding.LAGKV_EWORKSPACE
+    ws = plan.new_workspace()
+    with pytest.raises(binding.LagKVError) as e:      # misaligned cache pointer
+        plan.compress_prefill(K.view(-1)[1:1 + 2 * 299 * 128].view(1, 2, 299, 128), V, ws, S_in=299)
+    assert e.value.code == binding.LAGKV_EINVAL
+    with pytest.raises(binding.LagKVError) as e:      # output aliases input
+        plan.compress_prefill(K, V, ws, out={"K_out": K, "V_out": V})
+    assert e.value.code == binding.LAGKV_EINVAL
+    assert plan.read_status(ws)[0] == 0
