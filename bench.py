@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the LagKV prefill compress pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one whole compress pass (partition, lag statistics, normalise + std, softmax,
+K+V sum, per-head top-k, compaction, sink and window copy) over every layer of one
+synthetic cache, issued as ONE kernel launch with the layers folded into the batch
+dimension.  The metric is compressed tokens*heads per second,
+layers*B*H_kv*Ls / time-per-pass, with inputs resident in HBM; ``e2e`` is the same metric
+with the cache starting and the compacted result ending in pinned host memory.  One JSON
+line is printed by rank 0.  With N > 1 every rank compresses its own cache of the same
+shape (independent sequences, no collective on the data path): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "compressed_tokens_heads_per_s"
+UNIT = "tokens*heads/s"
+DEFAULT_WORKLOAD = "llama8b_128k"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the stream kernel, from the ncu
+# capture summarised under profiles/ (captured on a smaller case of the same kernel and
+# scaled by processed units where noted there); None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def algorithmic_bytes(w, L_R: int) -> int:
+    """Every input row read once, every output row written once, index list written once."""
+    units = w.layers * w.B * w.H
+    return units * ((w.S + L_R) * 2 * w.D * 2 + 4 * L_R)
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples taken while the timed region runs."""
+    Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self, t0: float, t1: float) -> dict:
+        import datetime
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.proc.wait()
+        self.tmp.flush()
+        rows = Path(self.tmp.name).read_text().splitlines()
+        os.unlink(self.tmp.name)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        allrows = []
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 10:
+                continue
+            try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rec = (ts, float(f[2]), float(f[3]), float(f[4]), f[6:10])
+            except ValueError:
+                continue
+            allrows.append(rec)
+        inside = [r for r in allrows if t0 - 0.05 <= r[0] <= t1 + 0.05] or allrows[-3:]
+        for ts, a, b, p, fl in inside:
+            sm.append(a)
+            smax.append(b)
+            power.append(p)
+            for n, v in zip(names, fl):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "reasons": sorted(reasons), "samples": len(inside)}
+
+
+def time_oracle(w, seconds_target: float = 12.0, layer_cap: int = 8):
+    """The oracle as it stands, timed on the host cores on whole layers of the workload."""
+    import numpy as np
+    from oracle import lagkv_oracle
+    from paper_2504_04704_b200 import synth
+    lagkv_oracle.build()
+    k = lagkv_oracle.keep_count(w.ratio, w.lag)
+    cores = lagkv_oracle.num_threads()
+    done_layers, spent = 0, 0.0
+    while done_layers < layer_cap:
+        K, V = synth.make_workload_layer(w, done_layers % w.layers, device="cpu")
+        Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+        del K, V
+        t0 = time.perf_counter()
+        lagkv_oracle.compress(Kb, Vb, w.sink, w.lag, k, want_scores=False)
+        spent += time.perf_counter() - t0
+        done_layers += 1
+        if spent + spent / done_layers > seconds_target * 1.5 or spent >= seconds_target:
+            break
+    th = done_layers * w.B * w.H * w.S
+    return {"value": th / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{done_layers} whole-layer passes (of the {w.layers} layers) of {w.name} "
+                      f"(B={w.B}, H={w.H}, Ls={w.S}), "
+                      f"{spent:.1f} s of float64 C with OpenMP", "seconds": spent, "tokens_heads": th}
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle on a bounded sample per step (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    vals = []
+    last = None
+    for i in range(args.warmup + args.steps):
+        last = time_oracle(w, seconds_target=per_step, layer_cap=4)
+        if i >= args.warmup:
+            vals.append(last)
+    tot_th = sum(v["tokens_heads"] for v in vals)
+    tot_s = sum(v["seconds"] for v in vals)
+    value = tot_th / tot_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / len(vals),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
+                   "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio,
+                   "note": "each step times the CPU oracle on a bounded sample of whole layers"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                         "sample": last["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a smaller case)")
+    ap.add_argument("--tune", default="", help="warps,tile_rows,stages,ctas_per_sm override")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    args = ap.parse_args()
+
+    from dataclasses import replace
+    from paper_2504_04704_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    if args.layers:
+        w = replace(w, layers=args.layers)
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__
+    from paper_2504_04704_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    binding.load_library()          # fails loudly if the CUDA library is missing
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    # ---- this rank's cache: all layers folded into the batch dimension, resident in HBM
+    Bf = w.layers * w.B
+    K = torch.empty((Bf, w.H, w.S, w.D), dtype=torch.bfloat16, device=dev)
+    V = torch.empty_like(K)
+    for layer in range(w.layers):
+        k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, w.seed(layer) + 100000 * rank, w.sigma_k, w.sigma_v, device=dev)
+        K[layer * w.B:(layer + 1) * w.B], V[layer * w.B:(layer + 1) * w.B] = k_l, v_l
+        del k_l, v_l
+    plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, device=local)
+    if args.tune:
+        t = [int(x) for x in args.tune.split(",")]
+        plan.tune(warps=t[0], tile_rows=t[1], stages=t[2], ctas_per_sm=t[3])
+    ws = plan.new_workspace()
+    L_R = plan.compressed_len(w.S)
+    out = {"K_out": torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, device=dev),
+           "V_out": torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, device=dev),
+           "idx": torch.empty((Bf, w.H, L_R), dtype=torch.int32, device=dev)}
+    info = plan.launch_info(w.S)
+    step = lambda: plan.compress_prefill(K, V, ws, out=out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert plan.read_status(ws)[0] == 0
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3 if rank == 0 else 0.0)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms_total = e0.elapsed_time(e1)
+    status = plan.read_status(ws)
+    assert status[0] == 0, f"device status {status}"
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    clocks = sampler.stop(wall0, wall1) if sampler else None
+    ms_step = ms_total / args.steps
+    units_per_rank = w.layers * w.B * w.H * w.S
+    value = world * units_per_rank / (ms_step * 1e-3)
+
+    # ---- end to end: host cache -> device -> compress -> compacted cache back on the host
+    e2e = None
+    if not args.no_e2e:
+        chunk = max(1, min(4, w.layers)) * w.B
+        while Bf % chunk:
+            chunk -= 1
+        del out
+        hp = binding.HostPrefill(Bf, w.H, w.D, w.S, w.sink, w.lag, keep_ratio=w.ratio, chunk_B=chunk, device=local)
+        Kh = torch.empty(K.shape, dtype=torch.bfloat16, pin_memory=True)
+        Vh = torch.empty(V.shape, dtype=torch.bfloat16, pin_memory=True)
+        Kh.copy_(K)
+        Vh.copy_(V)
+        Koh = torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, pin_memory=True)
+        Voh = torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, pin_memory=True)
+        Ih = torch.empty((Bf, w.H, L_R), dtype=torch.int32, pin_memory=True)
+        hp.run(Kh, Vh, Koh, Voh, Ih)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.e2e_steps):
+            hp.run(Kh, Vh, Koh, Voh, Ih)
+        f1.record(stream)
+        torch.cuda.synchronize()
+        ms_e2e = f0.elapsed_time(f1) / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * units_per_rank / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": hp.h2d_bytes, "d2h_bytes_per_step": hp.d2h_bytes, "steps": args.e2e_steps,
+               "chunk_layers": chunk // w.B}
+        del Kh, Vh, Koh, Voh, Ih, hp
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    alg = algorithmic_bytes(w, L_R)
+    achieved = alg / (ms_step * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get(w.name) if not args.layers else None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
+                   "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio, "keep_k": plan.k, "L_R": L_R,
+                   "storage": "bf16", "parallelism": f"dp{world} (independent caches per rank, no collective)",
+                   "launch": info, "l2": "inputs (%.1f GB per rank) are far larger than the 126 MB L2; no flush"
+                   % (2 * K.numel() * 2 / 1e9)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg,
+                     "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": "lagkv_stream_kernel"},
+        "clocks": clocks,
+        "gpu_launches": args.steps * info["launches"],
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu and world == 1:
+        del K, V
+        cb = time_oracle(w)
+        cb.pop("seconds"), cb.pop("tokens_heads")
+        line["cpu_baseline"] = cb
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

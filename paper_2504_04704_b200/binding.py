@@ -263,3 +263,66 @@ def lagkv_compress_append(plan: Plan, K_cache, V_cache, seq_len, static_len, wor
 
 def lagkv_gather(plan: Plan, K, V, idx, **kw):
     return plan.gather(K, V, idx, **kw)
+
+
+class HostPrefill:
+    """Prefill compression of a cache that lives in pinned HOST memory.
+
+    The ``[B, H, S_in, D]`` host cache is cut into chunks of ``chunk_B`` sequences (or
+    layers folded into B).  Each chunk is copied to a device staging buffer, compressed with
+    ``lagkv_compress_prefill`` and its compacted rows and indices are copied back; the three
+    stages run on three streams with two staging slots so that copies in both directions
+    overlap the kernel.  All arithmetic is the CUDA library's.
+    """
+
+    def __init__(self, B, H_kv, D, S_in, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1, chunk_B=1, device=0):
+        if B % chunk_B:
+            raise ValueError("B must be a multiple of chunk_B")
+        self.B, self.chunk_B, self.S_in = int(B), int(chunk_B), int(S_in)
+        self.plan = Plan(chunk_B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof,
+                         device=device)
+        dev = self.plan._dev()
+        self.L_R = self.plan.compressed_len(S_in)
+        self.ws = self.plan.new_workspace()
+        mk = lambda *shape, dt=torch.bfloat16: torch.empty(shape, dtype=dt, device=dev)
+        self.slots = [dict(K=mk(chunk_B, H_kv, S_in, D), V=mk(chunk_B, H_kv, S_in, D),
+                           K_out=mk(chunk_B, H_kv, self.L_R, D), V_out=mk(chunk_B, H_kv, self.L_R, D),
+                           idx=mk(chunk_B, H_kv, self.L_R, dt=torch.int32)) for _ in range(2)]
+        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream(dev) for _ in range(3))
+        self.h2d_bytes = 2 * B * H_kv * S_in * D * 2
+        self.d2h_bytes = 2 * B * H_kv * self.L_R * D * 2 + B * H_kv * self.L_R * 4
+
+    def run(self, K_host, V_host, K_out_host, V_out_host, idx_host) -> None:
+        """All five tensors are pinned host tensors; returns after the last copy has landed."""
+        cb = self.chunk_B
+        comp_done = [None, None]
+        out_done = [None, None]
+        cur = torch.cuda.current_stream(self.plan._dev())
+        for s in (self.s_in, self.s_comp, self.s_out):
+            s.wait_stream(cur)
+        for c in range(self.B // cb):
+            slot = self.slots[c % 2]
+            sl = slice(c * cb, (c + 1) * cb)
+            with torch.cuda.stream(self.s_in):
+                if comp_done[c % 2] is not None:
+                    self.s_in.wait_event(comp_done[c % 2])
+                slot["K"].copy_(K_host[sl], non_blocking=True)
+                slot["V"].copy_(V_host[sl], non_blocking=True)
+                in_done = torch.cuda.Event()
+                in_done.record(self.s_in)
+            with torch.cuda.stream(self.s_comp):
+                self.s_comp.wait_event(in_done)
+                if out_done[c % 2] is not None:
+                    self.s_comp.wait_event(out_done[c % 2])
+                self.plan.compress_prefill(slot["K"], slot["V"], self.ws, out=slot, want_scores=False)
+                comp_done[c % 2] = torch.cuda.Event()
+                comp_done[c % 2].record(self.s_comp)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(comp_done[c % 2])
+                K_out_host[sl].copy_(slot["K_out"], non_blocking=True)
+                V_out_host[sl].copy_(slot["V_out"], non_blocking=True)
+                idx_host[sl].copy_(slot["idx"], non_blocking=True)
+                out_done[c % 2] = torch.cuda.Event()
+                out_done[c % 2].record(self.s_out)
+        cur.wait_stream(self.s_out)
+        self.s_out.synchronize()

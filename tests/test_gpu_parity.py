@@ -346,7 +346,7 @@ def test_prefill_equals_incremental_on_gpu(binding, oracle):
 # ----------------------------------------------------------------------- argument checks
 def test_argument_errors(binding):
     with pytest.raises(binding.LagKVError) as e:
-        binding.Plan(1, 1, 100, 4, 64, device=0)
+        binding.Plan(1, 1, 96, 4, 64, device=0)
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
     with pytest.raises(binding.LagKVError) as e:
         binding.Plan(1, 1, 128, 4, 1, device=0)
