@@ -199,6 +199,7 @@ void lagkv_oracle_topk(const double *score, int64_t L, int64_t k, int32_t *idx_o
             if (taken[t]) continue;
             if (best < 0 || score[t] > score[best]) best = t; /* strict: lower index wins */
         }
+        if (best < 0) break; /* k > L: every token is already taken */
         taken[best] = 1;
     }
     int64_t w = 0;

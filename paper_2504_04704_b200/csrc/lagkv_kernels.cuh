@@ -165,6 +165,7 @@ struct SelScratch {
     int wsum[kMaxWarps];
     int bin;
     int krem;
+    int abort;  // set by a warp whose bounded wait ran out; the CTA stops at the next barrier
 };
 
 template <class G>
@@ -595,6 +596,7 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
     const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
     if (lane == 0)
         for (int i = 0; i < NS; ++i) mbar_init(bar_w + 8 * i, 1);
+    if (tid == 0) sc.abort = 0;
     fence_mbar_init();
     fence_proxy_async();
     __syncthreads();
@@ -634,7 +636,7 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
 
     int cslot = 0;
     uint32_t cparity = 0;
-    bool timed_out = false;
+    bool timed_out = false, aborted = false;
     const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
 
     f32x2 a2[G::NWORD], b2[G::NWORD];
@@ -656,17 +658,28 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
         float* sig = tensor ? sg1 : sg0;
 
         for (int t = wj; t < ntiles; t += G::WT) {
+            if (timed_out) break;  // nothing more is consumed once a wait has run out
             const uint32_t bar = bar_w + 8 * cslot;
-            if (!mbar_try_wait(bar, cparity)) {
+            // warp-uniform bounded wait: every lane polls, the warp moves on together, and
+            // lane 0's clock decides when to give up (about one second)
+            if (!__all_sync(0xffffffffu, mbar_try_wait(bar, cparity))) {
                 const unsigned long long t0 = global_timer_ns();
                 bool ok = false;
-                for (int it = 0; it < (1 << 26) && !ok; ++it) {
-                    ok = mbar_try_wait(bar, cparity);
-                    if (!ok && (it & 255) == 255 && global_timer_ns() - t0 > 1000000000ull) break;
+                for (int it = 0; it < (1 << 24); ++it) {
+                    ok = __all_sync(0xffffffffu, mbar_try_wait(bar, cparity));
+                    if (ok) break;
+                    if ((it & 255) == 255) {
+                        const int late = global_timer_ns() - t0 > 1000000000ull;
+                        if (__shfl_sync(0xffffffffu, late, 0)) break;
+                    }
                 }
                 if (!ok) {
                     timed_out = true;
-                    if (lane == 0) record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+                    if (lane == 0) {
+                        record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+                        *reinterpret_cast<volatile int*>(&sc.abort) = 1;
+                    }
+                    break;
                 }
             }
             const uint4* tile = reinterpret_cast<const uint4*>(ring + size_t(warp) * NS * G::TILE_BYTES +
@@ -708,6 +721,8 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
                 }
         }
         __syncthreads();
+        aborted = *reinterpret_cast<volatile int*>(&sc.abort) != 0;
+        if (aborted) break;  // uniform: every thread reads the flag after the same barrier
 
         // ---- select and emit partition p
         if (score) {
@@ -785,7 +800,7 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
     }
 
     // ---- append: pack kept rows behind the static part, then slide the window down
-    if (P.mode == MODE_APPEND) {
+    if (P.mode == MODE_APPEND && !aborted) {
         const int u = unit_fixed;
         uint16_t* ck = const_cast<uint16_t*>(unit_base(P.K, u));
         uint16_t* cv = const_cast<uint16_t*>(unit_base(P.V, u));
