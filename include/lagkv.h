@@ -178,10 +178,13 @@ int lagkv_read_status(lagkv_plan_t plan, void *workspace, void *cuda_stream,
 int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]);
 
 /*
- * Tuning override: warps per CTA (2, 4 or 8), rows per staged tile (16 or 32), ring
- * stages per warp (2..8) and resident CTAs per SM to size the grid for (>= 1).  A value
- * of 0 keeps the planner's choice.  Returns LAGKV_EUNSUPPORTED for a combination that was
- * not compiled or does not fit shared memory.
+ * Tuning override of the launch shape: warps per CTA (2, 4 or 8 = the uniform kernel, used
+ * for prefill and append alike; 12 = the warp-specialised prefill kernel with 8 streaming,
+ * 3 select and 1 copy warp, which leaves the append shape alone), rows per staged tile
+ * (16 or 32), ring stages per streaming warp (2..8) and resident CTAs per SM to size the
+ * prefill grid for (>= 1; must be 1 with 12 warps).  A value of 0 keeps the current
+ * choice.  Returns LAGKV_EUNSUPPORTED for a combination that was not compiled or does not
+ * fit shared memory.
  */
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages,
                     int32_t ctas_per_sm);

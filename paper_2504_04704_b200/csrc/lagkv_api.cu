@@ -9,6 +9,7 @@
 #include <new>
 
 #include "lagkv_kernels.cuh"
+#include "lagkv_ws_kernel.cuh"
 
 using namespace lagkv;
 
@@ -17,14 +18,19 @@ namespace {
 typedef void (*stream_kernel_t)(const Params);
 typedef size_t (*smem_fn_t)(int, int);
 
+// NW counts every warp of the CTA.  ws = warp-specialised prefill kernel (8 streaming
+// warps + 4 epilogue warps); the others are the uniform kernel that also serves appends.
 struct KernelEntry {
     int D, NW, TR;
+    bool ws;
     stream_kernel_t fn;
     smem_fn_t smem;
 };
 
 #define LAGKV_ENTRY(D, V, NW, TR) \
-    { D, NW, TR, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+    { D, NW, TR, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+#define LAGKV_WS_ENTRY(D, V, TR) \
+    { D, 8 + kWsEpiWarps, TR, true, &lagkv_ws_kernel<Geo<D, V, 8, TR>>, &ws_smem_total_bytes<Geo<D, V, 8, TR>> }
 
 const KernelEntry kKernels[] = {
     LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
@@ -33,6 +39,8 @@ const KernelEntry kKernels[] = {
     LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
     LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
     LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+    LAGKV_WS_ENTRY(128, 2, 32), LAGKV_WS_ENTRY(128, 2, 16), LAGKV_WS_ENTRY(64, 1, 32), LAGKV_WS_ENTRY(64, 1, 16),
+    LAGKV_WS_ENTRY(256, 2, 16),
 };
 constexpr int kNumKernels = int(sizeof(kKernels) / sizeof(kKernels[0]));
 
@@ -46,15 +54,20 @@ constexpr int kSmemPerSm = 233472;  // 228 KiB per SM, 1 KiB reserved per reside
 
 }  // namespace
 
+struct Shape {
+    int kidx;         // index into kKernels
+    int stages;       // ring depth per streaming warp
+    int ctas_per_sm;  // grid sizing for prefill
+    size_t smem;      // dynamic shared memory
+};
+
 struct lagkv_plan_s {
     lagkv_config cfg;
     int k;
     int sm_count;
     int max_smem_optin;
-    int kidx;         // index into kKernels
-    int stages;       // ring depth per warp
-    int ctas_per_sm;  // grid sizing for prefill
-    size_t smem;      // dynamic shared memory of the chosen kernel
+    Shape pre;        // kernel used by lagkv_compress_prefill
+    Shape app;        // kernel used by lagkv_compress_append (always the uniform kernel)
 };
 
 namespace {
@@ -80,10 +93,11 @@ int keep_count(double r, int L) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Try one launch shape; fills the plan fields on success.
-int apply_shape(lagkv_plan_s* pl, int NW, int TR, int stages, int ctas) {
+// Try one launch shape (NW = warps per CTA, 12 = the warp-specialised kernel).
+int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Shape* out) {
     const int kidx = find_kernel(pl->cfg.D, NW, TR);
     if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
+    if (kKernels[kidx].ws && ctas != 1) return LAGKV_EUNSUPPORTED;
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
     if (smem > size_t(pl->max_smem_optin)) return LAGKV_EUNSUPPORTED;
     if ((smem + 1024) * size_t(ctas) > size_t(kSmemPerSm)) return LAGKV_EUNSUPPORTED;
@@ -91,38 +105,56 @@ int apply_shape(lagkv_plan_s* pl, int NW, int TR, int stages, int ctas) {
         cudaFuncSetAttribute(reinterpret_cast<const void*>(kKernels[kidx].fn),
                              cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return LAGKV_ECUDA;
-    pl->kidx = kidx;
-    pl->stages = stages;
-    pl->ctas_per_sm = ctas;
-    pl->smem = smem;
+    out->kidx = kidx;
+    out->stages = stages;
+    out->ctas_per_sm = ctas;
+    out->smem = smem;
     return LAGKV_OK;
 }
 
-// Planner default: more warps and deeper rings for long partitions, many small CTAs for
-// short ones (the per-partition select phase is a fixed cost that other CTAs must hide).
-int choose_shape(lagkv_plan_s* pl) {
-    const int L = pl->cfg.lag;
-    struct Cand { int NW, TR, stages, ctas; };
-    Cand cands[8];
-    int nc = 0;
-    if (L >= 1024) {
-        cands[nc++] = {8, 32, 3, 1};
-        cands[nc++] = {8, 32, 2, 1};
-    }
-    if (L >= 256) {
-        cands[nc++] = {4, 32, 3, 2};
-        cands[nc++] = {4, 32, 2, 2};
-    }
-    cands[nc++] = {2, 16, 4, 6};
-    cands[nc++] = {2, 16, 3, 4};
-    cands[nc++] = {2, 16, 2, 2};
-    cands[nc++] = {2, 16, 2, 1};
+struct Cand {
+    int NW, TR, stages, ctas;
+};
+int first_fit(const lagkv_plan_s* pl, const Cand* cands, int nc, Shape* out) {
     int rc = LAGKV_EUNSUPPORTED;
     for (int i = 0; i < nc; ++i) {
-        rc = apply_shape(pl, cands[i].NW, cands[i].TR, cands[i].stages, cands[i].ctas);
+        rc = make_shape(pl, cands[i].NW, cands[i].TR, cands[i].stages, cands[i].ctas, out);
         if (rc == LAGKV_OK || rc == LAGKV_ECUDA) return rc;
     }
     return rc;
+}
+
+// Planner defaults.  Prefill: the warp-specialised kernel when partitions are long enough
+// to keep eight streaming warps busy, else many small uniform CTAs (the per-partition
+// select phase is a fixed cost that other CTAs must hide).  Append: uniform kernel, one
+// CTA per (b, h).
+int choose_shape(lagkv_plan_s* pl) {
+    const int L = pl->cfg.lag;
+    Cand uni[8];
+    int nu = 0;
+    if (L >= 1024) {
+        uni[nu++] = {8, 32, 3, 1};
+        uni[nu++] = {8, 32, 2, 1};
+    }
+    if (L >= 256) {
+        uni[nu++] = {4, 32, 3, 2};
+        uni[nu++] = {4, 32, 2, 2};
+    }
+    uni[nu++] = {2, 16, 4, 6};
+    uni[nu++] = {2, 16, 3, 4};
+    uni[nu++] = {2, 16, 2, 2};
+    uni[nu++] = {2, 16, 2, 1};
+    int rc = first_fit(pl, uni, nu, &pl->app);
+    if (rc != LAGKV_OK) return rc;
+    pl->pre = pl->app;
+    if (L >= 256) {
+        const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
+        Shape sh;
+        rc = first_fit(pl, ws, 3, &sh);
+        if (rc == LAGKV_ECUDA) return rc;
+        if (rc == LAGKV_OK) pl->pre = sh;
+    }
+    return LAGKV_OK;
 }
 
 struct Strides {
@@ -284,14 +316,14 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     P.rem = int(rest % c.lag);
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
     P.total_slots = U * P.n;
-    P.stages = plan->stages;
+    P.stages = plan->pre.stages;
 
-    const KernelEntry& ke = kKernels[plan->kidx];
-    long long grid = (long long)plan->sm_count * plan->ctas_per_sm;
+    const KernelEntry& ke = kKernels[plan->pre.kidx];
+    long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
     if (grid > P.total_slots) grid = P.total_slots;
     void* args[] = {&P};
     if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)grid), dim3(ke.NW * 32), args,
-                         plan->smem, stream) != cudaSuccess)
+                         plan->pre.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
     return check_launch();
 }
@@ -341,13 +373,13 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     P.S_in = int(S_cap);
     P.sink = c.sink;
     P.max_chunks = max_new_chunks;
-    P.stages = plan->stages;
+    P.stages = plan->app.stages;
 
-    const KernelEntry& ke = kKernels[plan->kidx];
+    const KernelEntry& ke = kKernels[plan->app.kidx];
     const long long U = (long long)c.B * c.H_kv;
     void* args[] = {&P};
     if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)U), dim3(ke.NW * 32), args,
-                         plan->smem, stream) != cudaSuccess)
+                         plan->app.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
     lagkv_update_lengths_kernel<<<(c.B + 127) / 128, 128, 0, stream>>>(seq_len, static_len, c.B, c.lag, plan->k,
                                                                        max_new_chunks, int(S_cap));
@@ -406,11 +438,11 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
         info[3] = S_in > 0 ? 1 : 0;
         return LAGKV_OK;
     }
-    long long grid = (long long)plan->sm_count * plan->ctas_per_sm;
+    long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
     const long long slots = U * (rest / c.lag);
     info[0] = int(grid < slots ? grid : slots);
-    info[1] = kKernels[plan->kidx].NW * 32;
-    info[2] = int(plan->smem);
+    info[1] = kKernels[plan->pre.kidx].NW * 32;
+    info[2] = int(plan->pre.smem);
     info[3] = 1;
     return LAGKV_OK;
 }
@@ -418,12 +450,15 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages, int32_t ctas_per_sm) {
     if (plan == nullptr) return LAGKV_EINVAL;
     DeviceGuard guard(plan->cfg.device);
-    const KernelEntry& cur = kKernels[plan->kidx];
-    lagkv_plan_s trial = *plan;
-    const int rc = apply_shape(&trial, warps ? warps : cur.NW, tile_rows ? tile_rows : cur.TR,
-                               stages ? stages : plan->stages, ctas_per_sm ? ctas_per_sm : plan->ctas_per_sm);
-    if (rc == LAGKV_OK) *plan = trial;
-    return rc;
+    const KernelEntry& cur = kKernels[plan->pre.kidx];
+    Shape sh;
+    const int rc = make_shape(plan, warps ? warps : cur.NW, tile_rows ? tile_rows : cur.TR,
+                              stages ? stages : plan->pre.stages, ctas_per_sm ? ctas_per_sm : plan->pre.ctas_per_sm,
+                              &sh);
+    if (rc != LAGKV_OK) return rc;
+    plan->pre = sh;
+    if (!kKernels[sh.kidx].ws) plan->app = sh;
+    return LAGKV_OK;
 }
 
 const char* lagkv_status_string(int status) {

@@ -78,6 +78,33 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         "l"(src), "r"(bytes), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// every bulk store committed by this thread has finished reading shared memory
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// barrier over `nthreads` threads (a multiple of 32) that all name the same id (1..15)
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// same barrier, returning the OR of `pred` over all participants
+__device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %3, 0;\n\t"
+        "bar.red.or.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"(uint32_t(pred))
+        : "memory");
+    return r != 0;
+}
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -88,6 +115,21 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
+}
+// Warp-collective bounded wait on an mbarrier phase: every lane polls, the warp leaves
+// together, and lane 0's clock decides when to give up (about one second).  Returns false
+// when the wait ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (int it = 0; it < (1 << 24); ++it) {
+        if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        if ((it & 255) == 255) {
+            const int late = global_timer_ns() - t0 > 1000000000ull;
+            if (__shfl_sync(0xffffffffu, late, 0)) break;
+        }
+    }
+    return false;
 }
 __device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
     uint32_t r;
@@ -264,9 +306,9 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
 // In: sg0 = sigma(K), sg1 = sigma(V), L entries each (shared memory).
 // Out: sg0 = final score (Eq. 11); kept = (int*)sg1 holds the k selected indices ascending.
 // All NT threads of the CTA must call; contains block barriers.
-template <int NT>
+template <int NT, class Sync>
 __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool single_tensor,
-                                 float* __restrict__ scores_g, SelScratch& sc, int tid) {
+                                 float* __restrict__ scores_g, SelScratch& sc, int tid, Sync sync) {
     constexpr int NWARP = NT / 32;
     const int lane = tid & 31, warp = tid >> 5;
 
@@ -286,7 +328,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
             sc.red[0][warp] = m0;
             sc.red[1][warp] = m1;
         }
-        __syncthreads();
+        sync();
         m0 = sc.red[0][0];
         m1 = sc.red[1][0];
 #pragma unroll
@@ -311,7 +353,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
             sc.red[2][warp] = s0;
             sc.red[3][warp] = s1;
         }
-        __syncthreads();
+        sync();
         s0 = sc.red[2][0];
         s1 = sc.red[3][0];
 #pragma unroll
@@ -328,14 +370,14 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
     } else if (scores_g != nullptr) {
         for (int t = tid; t < L; t += NT) scores_g[t] = sg0[t];
     }
-    __syncthreads();
+    sync();
 
     // ---- radix select: key of the k-th largest score, 8 bits per pass
     uint32_t prefix = 0, mask = 0;
     int krem = k;
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += NT) sc.hist[i] = 0;
-        __syncthreads();
+        sync();
         for (int t0 = 0; t0 < L; t0 += NT) {
             const int t = t0 + tid;
             const bool in = t < L;
@@ -346,7 +388,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
             const uint32_t peers = __match_any_sync(0xffffffffu, bin);
             if (act && lane == (__ffs(peers) - 1)) atomicAdd(&sc.hist[bin], __popc(peers));
         }
-        __syncthreads();
+        sync();
         if (warp == 0) {
             // lane owns bins [8*lane, 8*lane+8); walk from the top bin down
             int c[8], tot = 0;
@@ -374,7 +416,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
                 }
             }
         }
-        __syncthreads();
+        sync();
         prefix |= uint32_t(sc.bin) << shift;
         mask |= 255u << shift;
         krem = sc.krem;
@@ -397,7 +439,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
         if (lane >= o) incl += v;
     }
     if (lane == 31) sc.wsum[warp] = incl;
-    __syncthreads();  // also: every thread is done reading sg1, so kept[] may overwrite it
+    sync();  // also: every thread is done reading sg1, so kept[] may overwrite it
     int off = 0;
 #pragma unroll
     for (int w = 0; w < NWARP; ++w)
@@ -415,7 +457,7 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
             ++peq;
         }
     }
-    __syncthreads();
+    sync();
 }
 
 // --------------------------------------------------------------------------- row copies
@@ -458,14 +500,13 @@ __device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __r
 }
 
 // kept rows of one partition -> output (prefill, out of place)
-template <int NT, int VPR>
+template <int NT, int VPR, int U = 4>
 __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
                           long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
                           int src_row0, int dst_row0, const int* __restrict__ kept, int k,
                           int32_t* __restrict__ idx_dst, int tid) {
     if (dstK != nullptr) {
         const int items = k * 2 * VPR;
-        constexpr int U = 4;
         for (int base = 0; base < items; base += NT * U) {
             uint4 buf[U];
 #pragma unroll
@@ -660,27 +701,13 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
         for (int t = wj; t < ntiles; t += G::WT) {
             if (timed_out) break;  // nothing more is consumed once a wait has run out
             const uint32_t bar = bar_w + 8 * cslot;
-            // warp-uniform bounded wait: every lane polls, the warp moves on together, and
-            // lane 0's clock decides when to give up (about one second)
-            if (!__all_sync(0xffffffffu, mbar_try_wait(bar, cparity))) {
-                const unsigned long long t0 = global_timer_ns();
-                bool ok = false;
-                for (int it = 0; it < (1 << 24); ++it) {
-                    ok = __all_sync(0xffffffffu, mbar_try_wait(bar, cparity));
-                    if (ok) break;
-                    if ((it & 255) == 255) {
-                        const int late = global_timer_ns() - t0 > 1000000000ull;
-                        if (__shfl_sync(0xffffffffu, late, 0)) break;
-                    }
+            if (!mbar_wait_bounded(bar, cparity)) {
+                timed_out = true;
+                if (lane == 0) {
+                    record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+                    *reinterpret_cast<volatile int*>(&sc.abort) = 1;
                 }
-                if (!ok) {
-                    timed_out = true;
-                    if (lane == 0) {
-                        record_status(P.status, ST_ETIMEOUT, blockIdx.x);
-                        *reinterpret_cast<volatile int*>(&sc.abort) = 1;
-                    }
-                    break;
-                }
+                break;
             }
             const uint4* tile = reinterpret_cast<const uint4*>(ring + size_t(warp) * NS * G::TILE_BYTES +
                                                                size_t(cslot) * G::TILE_BYTES);
@@ -732,7 +759,7 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
                 scores_g = (P.mode == MODE_PREFILL)
                                ? P.scores_out + ((long long)u * n_c + p) * L
                                : P.scores_out + ((long long)u * P.max_chunks + p) * L;
-            score_and_select<G::NT>(sg0, sg1, L, k, false, scores_g, sc, tid);
+            score_and_select<G::NT>(sg0, sg1, L, k, false, scores_g, sc, tid, [] { __syncthreads(); });
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {
                 emit_kept<G::NT, G::VPR>(unit_base(P.K, u), unit_base(P.V, u), P.ss,

@@ -1,0 +1,370 @@
+// LagKV prefill compress pass -- warp-specialised persistent kernel for sm_100a.
+//
+// Same slot walk as lagkv_stream_kernel (partitions of a unit in DESCENDING p, so the
+// statistics of partition p+1, Eq. 7 / Eq. 8, are at hand when p streams through), but the
+// CTA is split into three roles so that the streaming never stops:
+//
+//   * NW streaming warps (even: K, odd: V).  Each owns a ring of shared-memory tiles
+//     filled by bulk async copies, normalises and accumulates the per-token moments
+//     (Eq. 9, Eq. 10) and the partition's own min / max, writes sigma into one of two
+//     sigma buffers and hands the slot over through an mbarrier.  The warps of one
+//     tensor meet once per partition on a named barrier to combine their min / max.
+//   * 3 select warps: softmax over the partition, K + V (Eq. 11), radix top-k with ties
+//     to the lower index, and the copy of the kept rows to the output -- one partition
+//     behind the streamers, overlapped with them.
+//   * 1 copy warp: the rows that are kept verbatim (sink and sliding window) of ALL
+//     units are cut into chunks dealt round-robin to the CTAs; the warp moves its chunks
+//     global -> shared -> global with bulk async copies, independent of the slot walk.
+//
+// Every wait on an mbarrier is bounded; a warp whose wait ran out raises the CTA's abort
+// flag, records LAGKV_ETIMEOUT and from then on only keeps the barrier protocol alive so
+// that no other warp blocks.
+#pragma once
+#include "lagkv_kernels.cuh"
+
+namespace lagkv {
+
+constexpr int kWsEpiWarps = 4;      // 3 select warps + 1 copy warp
+constexpr int kWsSelThreads = 96;
+constexpr int kWsCopyRows = 32;     // rows per staged chunk of the verbatim copies
+constexpr int kBarTensor = 1;       // named barriers 1, 2: streaming warps of K, of V
+constexpr int kBarSelect = 3;       // named barrier 3: the select warps
+
+template <class G>
+__host__ __device__ inline size_t ws_smem_total_bytes(int stages, int L) {
+    size_t s = smem_ring_bytes<G>(stages);                  // tile rings
+    s += size_t(2) * 2 * kWsCopyRows * G::D * 2;            // copy staging [2 stages][K, V]
+    s += (size_t(G::NW) * stages + 6) * 8;                  // mbarriers
+    s += size_t(2) * 2 * G::WT * 2 * (G::D / 2) * 4;        // min/max partials [2][K,V][WT][mn,mx]
+    s += sizeof(SelScratch);
+    s = (s + 15) & ~size_t(15);
+    s += size_t(2) * 2 * ((L + 3) & ~3) * 4;                // sigma [2 buffers][K, V]
+    return s + 128;                                         // alignment slack
+}
+
+template <class G>
+__global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(const Params P) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int NS = P.stages;
+    constexpr int CHUNK_BYTES = kWsCopyRows * G::D * 2;     // one tensor, one staged chunk
+    unsigned char* ring = sm;
+    unsigned char* stage = ring + smem_ring_bytes<G>(NS);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stage + 4 * CHUNK_BYTES);
+    uint64_t* xbars = bars + G::NW * NS;                    // full[2], empty[2], copy[2]
+    uint32_t* stats = reinterpret_cast<uint32_t*>(xbars + 6);
+    constexpr int STAT_WORDS = G::D / 2;                    // packed bf16x2 words per min (or max) row
+    SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * 2 * G::WT * 2 * STAT_WORDS);
+    float* sgbase = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
+    const int Lp = (P.L + 3) & ~3;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int L = P.L, k = P.k, n = P.n, sink = P.sink;
+    const int ntiles = (L + G::TR - 1) / G::TR;
+    const bool contiguous = (P.ss == G::D);
+
+    // slots [s_first, s_hi) belong to this CTA; a range that starts inside a unit first
+    // re-reads the partition above it (statistics only)
+    const long long s_first = P.total_slots * blockIdx.x / gridDim.x;
+    const long long s_hi = P.total_slots * (blockIdx.x + 1) / gridDim.x;
+    const bool extra = s_first < s_hi && (s_first % n) != 0;
+    const long long s_lo = extra ? s_first - 1 : s_first;
+
+    const uint32_t full_bar = smem_u32(xbars), empty_bar = smem_u32(xbars + 2), copy_bar = smem_u32(xbars + 4);
+    if (warp < G::NW && lane == 0)
+        for (int i = 0; i < NS; ++i) mbar_init(smem_u32(bars) + uint32_t(warp * NS + i) * 8, 1);
+    if (tid == 0) {
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(full_bar + 8 * b, G::NW);
+            mbar_init(empty_bar + 8 * b, 1);
+            mbar_init(copy_bar + 8 * b, 1);
+        }
+        sc.abort = 0;
+    }
+    fence_mbar_init();
+    fence_proxy_async();
+    __syncthreads();
+
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(&sc.abort);
+    auto raise_abort = [&]() {  // warp-collective
+        if (lane == 0) {
+            record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+            *abort_flag = 1;
+        }
+    };
+    auto unit_base = [&](const uint16_t* base, int u) -> const uint16_t* {
+        return base + (long long)(u / P.H) * P.sb + (long long)(u % P.H) * P.sh;
+    };
+
+    if (warp < G::NW) {
+        // =============================================================== streaming warps
+        const int tensor = warp & 1, wj = warp >> 1;
+        const int cg = lane % G::LPR, rl = lane / G::LPR;
+        const uint16_t* tbase = tensor ? P.V : P.K;
+        const uint32_t ring_w = smem_u32(ring) + uint32_t(warp) * NS * G::TILE_BYTES;
+        const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
+        bool dead = false;
+
+        const bool has_tiles = wj < ntiles;
+        long long ps = s_lo;  // producer cursor: next tile to request
+        int pt = wj, pslot = 0;
+        auto issue_next = [&]() {  // warp-collective
+            if (dead || !has_tiles || ps >= s_hi) return;
+            const int u = int(ps / n), p = n - 1 - int(ps % n);
+            const int row0 = sink + p * L + pt * G::TR;
+            const int rows = min(G::TR, L - pt * G::TR);
+            const uint16_t* src = unit_base(tbase, u) + (long long)row0 * P.ss;
+            const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
+            const uint32_t bar = bar_w + 8 * pslot;
+            const uint32_t bytes = uint32_t(rows) * G::D * 2;
+            if (lane == 0) {
+                fence_proxy_async();
+                mbar_arrive_expect_tx(bar, bytes);
+            }
+            if (contiguous) {
+                if (lane == 0) bulk_g2s(dst, src, bytes, bar);
+            } else {
+                __syncwarp();
+                for (int r = lane; r < rows; r += 32)
+                    bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+            }
+            pt += G::WT;
+            if (pt >= ntiles) {
+                pt = wj;
+                ++ps;
+            }
+            if (++pslot == NS) pslot = 0;
+        };
+        for (int i = 0; i < NS; ++i) issue_next();
+
+        int cslot = 0;
+        uint32_t cparity = 0;
+        const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
+        f32x2 a2[G::NWORD], b2[G::NWORD];
+#pragma unroll
+        for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
+
+        for (long long s = s_lo; s < s_hi; ++s) {
+            const int i = int(s - s_lo), buf = i & 1;
+            const int p = n - 1 - int(s % n);
+            const bool score = (p != n - 1) && s >= s_first;
+            dead = __any_sync(0xffffffffu, dead || *abort_flag != 0);
+            // the select warps must have released this sigma buffer (slot i - 2)
+            if (i >= 2 && !dead && !mbar_wait_bounded(empty_bar + 8 * buf, uint32_t((i >> 1) - 1) & 1u)) {
+                dead = true;
+                raise_abort();
+            }
+
+            uint32_t mn[G::NWORD], mx[G::NWORD];
+#pragma unroll
+            for (int j = 0; j < G::NWORD; ++j) {
+                mn[j] = 0x7f807f80u;  // +inf, +inf
+                mx[j] = 0xff80ff80u;  // -inf, -inf
+            }
+            float* sig = sgbase + (buf * 2 + tensor) * Lp;
+
+            for (int t = wj; t < ntiles; t += G::WT) {
+                if (dead) break;
+                if (!mbar_wait_bounded(bar_w + 8 * cslot, cparity)) {
+                    dead = true;
+                    raise_abort();
+                    break;
+                }
+                const uint4* tile = reinterpret_cast<const uint4*>(ring + size_t(warp) * NS * G::TILE_BYTES +
+                                                                   size_t(cslot) * G::TILE_BYTES);
+                const int nrows = min(G::TR, L - t * G::TR);
+                float* so = sig + t * G::TR;
+                if (nrows == G::TR) {
+                    if (score) process_tile<G, true, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                    else process_tile<G, false, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                } else {
+                    if (score) process_tile<G, true, false>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                    else process_tile<G, false, false>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
+                }
+                __syncwarp();
+                issue_next();  // refill the slot just drained
+                if (++cslot == NS) {
+                    cslot = 0;
+                    cparity ^= 1u;
+                }
+            }
+
+            // ---- this partition's min / max (Eq. 7, Eq. 8): lanes sharing channels, then warps
+#pragma unroll
+            for (int j = 0; j < G::NWORD; ++j) {
+#pragma unroll
+                for (int o = G::LPR; o < 32; o <<= 1) {
+                    mn[j] = bf2_min(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
+                    mx[j] = bf2_max(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+                }
+            }
+            uint32_t* stats_t = stats + ((buf * 2 + tensor) * G::WT) * 2 * STAT_WORDS;
+            if (rl == 0) {
+                uint32_t* st = stats_t + wj * 2 * STAT_WORDS;
+#pragma unroll
+                for (int v = 0; v < G::V; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        st[(v * G::LPR + cg) * 4 + c] = mn[v * 4 + c];
+                        st[STAT_WORDS + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
+                    }
+            }
+            named_bar_sync(kBarTensor + tensor, G::WT * 32);
+            // sigma of this tensor is complete: hand the slot to the select warps
+            if (lane == 0) mbar_arrive(full_bar + 8 * buf);
+
+            // ---- coefficients for the next (lower) partition from this one's statistics:
+            //      y = (z - mid) / range, a shift of Eq. 9 by -1/2 that leaves the std unchanged
+            {
+                uint32_t fmn[G::NWORD], fmx[G::NWORD];
+#pragma unroll
+                for (int j = 0; j < G::NWORD; ++j) {
+                    fmn[j] = 0x7f807f80u;
+                    fmx[j] = 0xff80ff80u;
+                }
+                for (int w = 0; w < G::WT; ++w) {
+                    const uint32_t* st = stats_t + w * 2 * STAT_WORDS;
+#pragma unroll
+                    for (int v = 0; v < G::V; ++v)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            fmn[v * 4 + c] = bf2_min(fmn[v * 4 + c], st[(v * G::LPR + cg) * 4 + c]);
+                            fmx[v * 4 + c] = bf2_max(fmx[v * 4 + c], st[STAT_WORDS + (v * G::LPR + cg) * 4 + c]);
+                        }
+                }
+                int zero_range = 0;
+#pragma unroll
+                for (int j = 0; j < G::NWORD; ++j) {
+                    const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
+                    const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
+                    const float r0 = hi0 - lo0, r1 = hi1 - lo1;
+                    const float a0 = r0 > 0.f ? 1.0f / r0 : 0.f, a1 = r1 > 0.f ? 1.0f / r1 : 0.f;
+                    const float c0 = r0 > 0.f ? -(0.5f * (lo0 + hi0)) * a0 : -0.5f;
+                    const float c1 = r1 > 0.f ? -(0.5f * (lo1 + hi1)) * a1 : -0.5f;
+                    zero_range += !(r0 > 0.f);
+                    zero_range += !(r1 > 0.f);
+                    a2[j] = pack2(a0, a1);
+                    b2[j] = pack2(c0, c1);
+                }
+                if (zero_range != 0 && wj == 0 && rl == 0 && !dead && P.status != nullptr)
+                    atomicAdd(P.status + 2, zero_range);
+            }
+        }
+        if (dead) {  // copies may still be in flight towards this CTA's shared memory
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
+        }
+    } else if (warp < G::NW + 3) {
+        // ================================================================== select warps
+        const int etid = tid - G::NT;
+        bool dead = false;
+        auto sync_sel = [] { named_bar_sync(kBarSelect, kWsSelThreads); };
+        for (long long s = s_lo; s < s_hi; ++s) {
+            const int i = int(s - s_lo), buf = i & 1;
+            const int u = int(s / n), p = n - 1 - int(s % n);
+            const bool score = (p != n - 1) && s >= s_first;
+            bool bad = __any_sync(0xffffffffu, dead || *abort_flag != 0);
+            if (!bad && !mbar_wait_bounded(full_bar + 8 * buf, uint32_t(i >> 1) & 1u)) {
+                bad = true;
+                raise_abort();
+            }
+            dead = named_bar_or(kBarSelect, kWsSelThreads, bad);  // one verdict for the group
+            if (score && !dead) {
+                float* sg0 = sgbase + (buf * 2) * Lp;
+                float* sg1 = sg0 + Lp;
+                float* scores_g = P.scores_out ? P.scores_out + ((long long)u * (n - 1) + p) * L : nullptr;
+                score_and_select<kWsSelThreads>(sg0, sg1, L, k, false, scores_g, sc, etid, sync_sel);
+                emit_kept<kWsSelThreads, G::VPR, 8>(
+                    unit_base(P.K, u), unit_base(P.V, u), P.ss,
+                    P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr,
+                    P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr, sink + p * L, sink + p * k,
+                    reinterpret_cast<const int*>(sg1), k, P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr,
+                    etid);
+                sync_sel();  // every thread is done with this sigma buffer
+            }
+            if (etid == 0) mbar_arrive(empty_bar + 8 * buf);
+        }
+    } else {
+        // ===================================================================== copy warp
+        // Chunks of the verbatim rows of every unit: first the window chunks, then the sink
+        // chunks of unit 0, then unit 1, ...; chunk g is handled by CTA g mod gridDim.x.
+        const int win_rows = L + P.rem;
+        const int cw = (win_rows + kWsCopyRows - 1) / kWsCopyRows, cs = (sink + kWsCopyRows - 1) / kWsCopyRows;
+        const long long U = (long long)P.B * P.H;
+        const long long total_chunks = U * (cw + cs);
+        const bool rows_wanted = P.K_out != nullptr;
+        const uint32_t stage_u32 = smem_u32(stage);
+        int pu = 0, pdst = 0, pnr = 0;  // chunk loaded in the previous round, not yet stored
+        bool pending = false, dead = false;
+        int round = 0;
+        for (long long g = blockIdx.x;; g += gridDim.x, ++round) {
+            const bool have = g < total_chunks;
+            if (!have && !pending) break;
+            const int st = round & 1;
+            int u = 0, src = 0, dst = 0, nr = 0;
+            if (have) {
+                u = int(g / (cw + cs));
+                const int j = int(g % (cw + cs));
+                if (j < cw) {
+                    src = sink + (n - 1) * L + j * kWsCopyRows;
+                    dst = sink + (n - 1) * k + j * kWsCopyRows;
+                    nr = min(kWsCopyRows, win_rows - j * kWsCopyRows);
+                } else {
+                    src = dst = (j - cw) * kWsCopyRows;
+                    nr = min(kWsCopyRows, sink - (j - cw) * kWsCopyRows);
+                }
+                if (P.idx_out != nullptr)
+                    for (int r = lane; r < nr; r += 32) P.idx_out[(long long)u * P.L_R + dst + r] = src + r;
+            }
+            if (rows_wanted && !dead) {
+                if (have) {
+                    // stage `st` was last read by the store committed two rounds ago
+                    if (lane == 0) {
+                        bulk_wait_read_all();
+                        fence_proxy_async();
+                        mbar_arrive_expect_tx(copy_bar + 8 * st, uint32_t(2 * nr) * G::D * 2);
+                    }
+                    __syncwarp();
+                    const uint32_t dK = stage_u32 + uint32_t(2 * st) * CHUNK_BYTES, dV = dK + CHUNK_BYTES;
+                    const uint16_t* sK = unit_base(P.K, u) + (long long)src * P.ss;
+                    const uint16_t* sV = unit_base(P.V, u) + (long long)src * P.ss;
+                    if (contiguous) {
+                        if (lane == 0) {
+                            bulk_g2s(dK, sK, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                            bulk_g2s(dV, sV, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                        }
+                    } else {
+                        for (int r = lane; r < nr; r += 32) {
+                            bulk_g2s(dK + uint32_t(r) * G::D * 2, sK + (long long)r * P.ss, G::D * 2, copy_bar + 8 * st);
+                            bulk_g2s(dV + uint32_t(r) * G::D * 2, sV + (long long)r * P.ss, G::D * 2, copy_bar + 8 * st);
+                        }
+                    }
+                }
+                if (pending) {  // the chunk loaded one round ago goes out
+                    const int pst = (round - 1) & 1;
+                    if (!mbar_wait_bounded(copy_bar + 8 * pst, uint32_t((round - 1) >> 1) & 1u)) {
+                        dead = true;
+                        raise_abort();
+                    } else if (lane == 0) {
+                        fence_proxy_async();
+                        const uint32_t sK = stage_u32 + uint32_t(2 * pst) * CHUNK_BYTES, sV = sK + CHUNK_BYTES;
+                        bulk_s2g(P.K_out + ((long long)pu * P.L_R + pdst) * G::D, sK, uint32_t(pnr) * G::D * 2);
+                        bulk_s2g(P.V_out + ((long long)pu * P.L_R + pdst) * G::D, sV, uint32_t(pnr) * G::D * 2);
+                        bulk_commit();
+                    }
+                }
+            }
+            pending = have;
+            pu = u;
+            pdst = dst;
+            pnr = nr;
+        }
+        if (lane == 0) bulk_wait_read_all();
+        if (dead) {
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
+        }
+    }
+}
+
+}  // namespace lagkv

@@ -136,17 +136,32 @@ def test_prefill_strided_layouts(binding, oracle, layout):
 
 
 @pytest.mark.parametrize("warps,tile_rows,stages", [(8, 32, 3), (8, 32, 2), (4, 32, 4), (2, 32, 3), (8, 16, 4),
-                                                    (4, 16, 2), (2, 16, 8)])
+                                                    (4, 16, 2), (2, 16, 8), (12, 32, 2), (12, 16, 3), (12, 16, 2)])
 def test_prefill_every_launch_shape(binding, oracle, warps, tile_rows, stages):
     run_prefill(binding, oracle, 1, 6, 128, 16 + 7 * 320 + 100, 16, 320, 80, seed=warps * 100 + tile_rows + stages,
                 tune=dict(warps=warps, tile_rows=tile_rows, stages=stages, ctas_per_sm=1))
 
 
-def test_prefill_many_units_ranges_start_mid_unit(binding, oracle):
+@pytest.mark.parametrize("warps,tile_rows,stages", [(2, 16, 3), (12, 32, 2)])
+def test_prefill_many_units_ranges_start_mid_unit(binding, oracle, warps, tile_rows, stages):
     """More (b, h) units than CTAs and a partition count that does not divide evenly, so
     CTA ranges begin inside units and re-read a reference partition."""
-    run_prefill(binding, oracle, 7, 5, 128, 3 + 6 * 64 + 5, 3, 64, 16, seed=77,
-                tune=dict(warps=2, tile_rows=16, stages=3, ctas_per_sm=1))
+    run_prefill(binding, oracle, 37, 5, 128, 3 + 6 * 64 + 5, 3, 64, 16, seed=77,
+                tune=dict(warps=warps, tile_rows=tile_rows, stages=stages, ctas_per_sm=1))
+
+
+@pytest.mark.parametrize("L,k,S_extra", [(64, 4, 60), (100, 25, 7), (72, 72, 0), (256, 1, 255), (37, 5, 36), (2, 1, 1)])
+def test_prefill_warp_specialised_short_partitions(binding, oracle, L, k, S_extra):
+    """The warp-specialised kernel forced onto partitions shorter than its default range
+    (fewer tiles than streaming warps, ragged tiles, sink shorter than a copy chunk)."""
+    run_prefill(binding, oracle, 2, 3, 128, 4 + 9 * L + S_extra, 4, L, k, seed=L + 1,
+                tune=dict(warps=12, tile_rows=32, stages=2, ctas_per_sm=1))
+
+
+@pytest.mark.parametrize("layout", ["bshd", "padded"])
+def test_prefill_warp_specialised_strided(binding, oracle, layout):
+    run_prefill(binding, oracle, 2, 4, 128, 40 + 4 * 300 + 111, 40, 300, 75, seed=4, layout=layout,
+                tune=dict(warps=12, tile_rows=32, stages=2, ctas_per_sm=1))
 
 
 def test_prefill_heavy_outliers(binding, oracle):

@@ -89,7 +89,7 @@ def test_launch_shapes_fit_the_sm(binding):
     for L in (64, 128, 256, 512, 1024, 2048, 4096, 8192):
         plan = binding.Plan(32, 8, 128, 16, L, device=-1)
         info = plan.launch_info(16 + 40 * L)
-        assert info["smem"] <= 232448 and info["block"] in (64, 128, 256) and info["grid"] >= 148
+        assert info["smem"] <= 232448 and info["block"] in (64, 128, 256, 384) and info["grid"] >= 148
     plan = binding.Plan(1, 8, 128, 16, 128, device=-1)
     assert plan.launch_info(100)["smem"] == 0        # identity pass: plain copy kernel
     with pytest.raises(binding.LagKVError):
