@@ -105,6 +105,10 @@ __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
         : "memory");
     return r != 0;
 }
+// ask L2 to fetch `bytes` (a multiple of 16, 16-byte aligned address) of global memory
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -202,7 +206,9 @@ struct Geo {
 };
 
 struct SelScratch {
-    float red[4][kMaxWarps];
+    unsigned long long redq[2][kMaxWarps];
+    float red[2][kMaxWarps];
+    int cnt[2][kMaxWarps];
     int hist[256];
     int wsum[kMaxWarps];
     int bin;
@@ -303,72 +309,212 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
 }
 
 // -------------------------------------------------------------- softmax + top-k (block)
-// In: sg0 = sigma(K), sg1 = sigma(V), L entries each (shared memory).
-// Out: sg0 = final score (Eq. 11); kept = (int*)sg1 holds the k selected indices ascending.
-// All NT threads of the CTA must call; contains block barriers.
-template <int NT, class Sync>
-__device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool single_tensor,
-                                 float* __restrict__ scores_g, SelScratch& sc, int tid, Sync sync) {
+// The softmax denominators are accumulated as integers (exp value times 2^40, rounded), so
+// they do not depend on which thread adds what: the scores, and with them the selection,
+// are a function of the sigma values alone, bit-identical for every launch shape and for
+// both implementations below.
+__device__ __forceinline__ unsigned long long fx40(float e) { return __float2ull_rn(e * 1099511627776.0f); }
+__device__ __forceinline__ float fx40_to_float(unsigned long long q) {
+    return __ull2float_rn(q) * (1.0f / 1099511627776.0f);
+}
+// Eq. 11 from the two exponentials and the two softmax denominators
+__device__ __forceinline__ float combine_scores(float e0, float s0, float e1, float s1) {
+    return __fadd_rn(__fdiv_rn(e0, s0), __fdiv_rn(e1, s1));
+}
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Both selectors: in sg0 = sigma(K), sg1 = sigma(V), L entries each (shared memory); out
+// kept[0..k) = the selected indices ascending (kept may alias sg1), scores_g (global, may
+// be null) = final scores.  All NT threads of the group call with group-local tid; sync()
+// is a barrier over exactly those NT threads; release() is called by every thread once no
+// thread of the group reads sg0 / sg1 any more (it may hand the buffers to a producer).
+
+// Selector for L <= NT * E: every thread keeps E consecutive tokens in registers; the key of
+// the k-th largest score is built bit by bit from block-wide counts.
+template <int NT, int E, class Sync, class Release>
+__device__ void select_in_registers(const float* sg0, const float* sg1, int L, int k,
+                                    float* __restrict__ scores_g, int* kept, SelScratch& sc, int tid, Sync sync,
+                                    Release release) {
+    constexpr int NWARP = NT / 32;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int t_lo = tid * E;
+    float x0[E], x1[E];
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        const int t = t_lo + j;
+        x0[j] = t < L ? sg0[t] : -INFINITY;
+        x1[j] = t < L ? sg1[t] : -INFINITY;
+        m0 = fmaxf(m0, x0[j]);
+        m1 = fmaxf(m1, x1[j]);
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+    }
+    if (lane == 0) {
+        sc.red[0][warp] = m0;
+        sc.red[1][warp] = m1;
+    }
+    sync();
+    release();
+    m0 = sc.red[0][0];
+    m1 = sc.red[1][0];
+#pragma unroll
+    for (int w = 1; w < NWARP; ++w) {
+        m0 = fmaxf(m0, sc.red[0][w]);
+        m1 = fmaxf(m1, sc.red[1][w]);
+    }
+    // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
+    unsigned long long q0 = 0, q1 = 0;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        x0[j] = expf(x0[j] - m0);  // exp(-inf) = 0 for the padding
+        x1[j] = expf(x1[j] - m1);
+        q0 += fx40(x0[j]);
+        q1 += fx40(x1[j]);
+    }
+    q0 = warp_sum_u64(q0);
+    q1 = warp_sum_u64(q1);
+    if (lane == 0) {
+        sc.redq[0][warp] = q0;
+        sc.redq[1][warp] = q1;
+    }
+    sync();
+    q0 = q1 = 0;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) {
+        q0 += sc.redq[0][w];
+        q1 += sc.redq[1][w];
+    }
+    const float s0 = fx40_to_float(q0), s1 = fx40_to_float(q1);
+    // ---- Eq. 11, then the order-preserving integer image; padding gets the smallest key
+    uint32_t key[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        const int t = t_lo + j;
+        const float sco = combine_scores(x0[j], s0, x1[j], s1);
+        key[j] = t < L ? float_key(sco) : 0u;
+        if (scores_g != nullptr && t < L) scores_g[t] = sco;
+    }
+    // ---- T = key of the k-th largest score: the largest T with count(key >= T) >= k
+    uint32_t T = 0;
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = T | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int j = 0; j < E; ++j) c += key[j] >= cand;
+        c = __reduce_add_sync(0xffffffffu, c);
+        const int par = bit & 1;
+        if (lane == 0) sc.cnt[par][warp] = c;
+        sync();
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) tot += sc.cnt[par][w];
+        if (tot >= k) T = cand;
+    }
+    // ---- positions: tokens above T all stay; of those equal to T the first krem
+    int cgt = 0, ceq = 0;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        cgt += key[j] > T;
+        ceq += key[j] == T;
+    }
+    const int packed = cgt | (ceq << 16);
+    int incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) sc.wsum[warp] = incl;
+    sync();
+    int off = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) {
+        const int ws = sc.wsum[w];
+        if (w < warp) off += ws;
+        total += ws;
+    }
+    const int krem = k - (total & 0xffff);
+    const int excl = off + incl - packed;
+    int pgt = excl & 0xffff, peq = excl >> 16;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        if (key[j] > T) {
+            kept[pgt + min(peq, krem)] = t_lo + j;
+            ++pgt;
+        } else if (key[j] == T) {
+            if (peq < krem) kept[pgt + peq] = t_lo + j;
+            ++peq;
+        }
+    }
+    sync();
+}
+
+// Selector for any L: scores stay in shared memory (sg0 is overwritten with them), radix
+// select with 8 bits per pass.
+template <int NT, class Sync, class Release>
+__device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __restrict__ scores_g, int* kept,
+                                 SelScratch& sc, int tid, Sync sync, Release release) {
     constexpr int NWARP = NT / 32;
     const int lane = tid & 31, warp = tid >> 5;
 
-    if (!single_tensor) {
-        // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
-        float m0 = -INFINITY, m1 = -INFINITY;
-        for (int t = tid; t < L; t += NT) {
-            m0 = fmaxf(m0, sg0[t]);
-            m1 = fmaxf(m1, sg1[t]);
-        }
+    // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
+    float m0 = -INFINITY, m1 = -INFINITY;
+    for (int t = tid; t < L; t += NT) {
+        m0 = fmaxf(m0, sg0[t]);
+        m1 = fmaxf(m1, sg1[t]);
+    }
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
-            m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
-        }
-        if (lane == 0) {
-            sc.red[0][warp] = m0;
-            sc.red[1][warp] = m1;
-        }
-        sync();
-        m0 = sc.red[0][0];
-        m1 = sc.red[1][0];
+    for (int o = 16; o >= 1; o >>= 1) {
+        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+    }
+    if (lane == 0) {
+        sc.red[0][warp] = m0;
+        sc.red[1][warp] = m1;
+    }
+    sync();
+    m0 = sc.red[0][0];
+    m1 = sc.red[1][0];
 #pragma unroll
-        for (int w = 1; w < NWARP; ++w) {
-            m0 = fmaxf(m0, sc.red[0][w]);
-            m1 = fmaxf(m1, sc.red[1][w]);
-        }
-        float s0 = 0.f, s1 = 0.f;
-        for (int t = tid; t < L; t += NT) {
-            const float e0 = expf(sg0[t] - m0), e1 = expf(sg1[t] - m1);
-            sg0[t] = e0;
-            sg1[t] = e1;
-            s0 += e0;
-            s1 += e1;
-        }
+    for (int w = 1; w < NWARP; ++w) {
+        m0 = fmaxf(m0, sc.red[0][w]);
+        m1 = fmaxf(m1, sc.red[1][w]);
+    }
+    unsigned long long q0 = 0, q1 = 0;
+    for (int t = tid; t < L; t += NT) {
+        const float e0 = expf(sg0[t] - m0), e1 = expf(sg1[t] - m1);
+        sg0[t] = e0;
+        sg1[t] = e1;
+        q0 += fx40(e0);
+        q1 += fx40(e1);
+    }
+    q0 = warp_sum_u64(q0);
+    q1 = warp_sum_u64(q1);
+    if (lane == 0) {
+        sc.redq[0][warp] = q0;
+        sc.redq[1][warp] = q1;
+    }
+    sync();
+    q0 = q1 = 0;
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-        }
-        if (lane == 0) {
-            sc.red[2][warp] = s0;
-            sc.red[3][warp] = s1;
-        }
-        sync();
-        s0 = sc.red[2][0];
-        s1 = sc.red[3][0];
-#pragma unroll
-        for (int w = 1; w < NWARP; ++w) {
-            s0 += sc.red[2][w];
-            s1 += sc.red[3][w];
-        }
-        // ---- Eq. 11
-        for (int t = tid; t < L; t += NT) {
-            const float s = sg0[t] / s0 + sg1[t] / s1;
-            sg0[t] = s;
-            if (scores_g != nullptr) scores_g[t] = s;
-        }
-    } else if (scores_g != nullptr) {
-        for (int t = tid; t < L; t += NT) scores_g[t] = sg0[t];
+    for (int w = 0; w < NWARP; ++w) {
+        q0 += sc.redq[0][w];
+        q1 += sc.redq[1][w];
+    }
+    const float s0 = fx40_to_float(q0), s1 = fx40_to_float(q1);
+    // ---- Eq. 11
+    for (int t = tid; t < L; t += NT) {
+        const float sco = combine_scores(sg0[t], s0, sg1[t], s1);
+        sg0[t] = sco;
+        if (scores_g != nullptr) scores_g[t] = sco;
     }
     sync();
 
@@ -446,7 +592,6 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
         if (w < warp) off += sc.wsum[w];
     const int excl = off + incl - packed;
     int pgt = excl & 0xffff, peq = excl >> 16;
-    int* kept = reinterpret_cast<int*>(sg1);
     for (int t = t_lo; t < t_hi; ++t) {
         const uint32_t key = float_key(sg0[t]);
         if (key > prefix) {
@@ -458,6 +603,17 @@ __device__ void score_and_select(float* sg0, float* sg1, int L, int k, bool sing
         }
     }
     sync();
+    release();
+}
+
+// Dispatch: registers when the partition fits E tokens per thread, else shared memory.
+template <int NT, class Sync, class Release>
+__device__ __forceinline__ void score_and_select(float* sg0, float* sg1, int L, int k,
+                                                 float* __restrict__ scores_g, int* kept, SelScratch& sc, int tid,
+                                                 Sync sync, Release release) {
+    if (L <= NT * 8) select_in_registers<NT, 8>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    else if (L <= NT * 22) select_in_registers<NT, 22>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    else select_in_shared<NT>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
 }
 
 // --------------------------------------------------------------------------- row copies
@@ -500,12 +656,18 @@ __device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __r
 }
 
 // kept rows of one partition -> output (prefill, out of place)
-template <int NT, int VPR, int U = 4>
+template <int NT, int VPR, int U = 4, bool PREFETCH = false>
 __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
                           long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
                           int src_row0, int dst_row0, const int* __restrict__ kept, int k,
                           int32_t* __restrict__ idx_dst, int tid) {
     if (dstK != nullptr) {
+        if (PREFETCH) {  // put every kept row in flight towards L2 before the first load waits
+            for (int j = tid; j < 2 * k; j += NT) {
+                const uint16_t* s = (j & 1) ? srcV : srcK;
+                prefetch_l2(s + (long long)(src_row0 + kept[j >> 1]) * ss, VPR * 16);
+            }
+        }
         const int items = k * 2 * VPR;
         for (int base = 0; base < items; base += NT * U) {
             uint4 buf[U];
@@ -759,7 +921,8 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
                 scores_g = (P.mode == MODE_PREFILL)
                                ? P.scores_out + ((long long)u * n_c + p) * L
                                : P.scores_out + ((long long)u * P.max_chunks + p) * L;
-            score_and_select<G::NT>(sg0, sg1, L, k, false, scores_g, sc, tid, [] { __syncthreads(); });
+            score_and_select<G::NT>(sg0, sg1, L, k, scores_g, reinterpret_cast<int*>(sg1), sc, tid,
+                                     [] { __syncthreads(); }, [] {});
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {
                 emit_kept<G::NT, G::VPR>(unit_base(P.K, u), unit_base(P.V, u), P.ss,

@@ -9,12 +9,15 @@
 //     (Eq. 9, Eq. 10) and the partition's own min / max, writes sigma into one of two
 //     sigma buffers and hands the slot over through an mbarrier.  The warps of one
 //     tensor meet once per partition on a named barrier to combine their min / max.
-//   * 3 select warps: softmax over the partition, K + V (Eq. 11), radix top-k with ties
-//     to the lower index, and the copy of the kept rows to the output -- one partition
-//     behind the streamers, overlapped with them.
+//   * 3 select warps: softmax over the partition, K + V (Eq. 11) and top-k with ties to
+//     the lower index -- one partition behind the streamers, overlapped with them.  They
+//     record where the kept rows come from; the rows move in the gather phase below.
 //   * 1 copy warp: the rows that are kept verbatim (sink and sliding window) of ALL
 //     units are cut into chunks dealt round-robin to the CTAs; the warp moves its chunks
 //     global -> shared -> global with bulk async copies, independent of the slot walk.
+//
+// When a CTA has walked all its slots, all of its warps together copy the kept rows of its
+// partitions to the output (gather phase).
 //
 // Every wait on an mbarrier is bounded; a warp whose wait ran out raises the CTA's abort
 // flag, records LAGKV_ETIMEOUT and from then on only keeps the barrier protocol alive so
@@ -39,6 +42,7 @@ __host__ __device__ inline size_t ws_smem_total_bytes(int stages, int L) {
     s += sizeof(SelScratch);
     s = (s + 15) & ~size_t(15);
     s += size_t(2) * 2 * ((L + 3) & ~3) * 4;                // sigma [2 buffers][K, V]
+    s += size_t((L + 3) & ~3) * 4;                          // kept indices of one partition
     return s + 128;                                         // alignment slack
 }
 
@@ -57,6 +61,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * 2 * G::WT * 2 * STAT_WORDS);
     float* sgbase = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
     const int Lp = (P.L + 3) & ~3;
+    int* kept = reinterpret_cast<int*>(sgbase + 4 * Lp);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = P.L, k = P.k, n = P.n, sink = P.sink;
@@ -273,16 +278,29 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 float* sg0 = sgbase + (buf * 2) * Lp;
                 float* sg1 = sg0 + Lp;
                 float* scores_g = P.scores_out ? P.scores_out + ((long long)u * (n - 1) + p) * L : nullptr;
-                score_and_select<kWsSelThreads>(sg0, sg1, L, k, false, scores_g, sc, etid, sync_sel);
-                emit_kept<kWsSelThreads, G::VPR, 8>(
-                    unit_base(P.K, u), unit_base(P.V, u), P.ss,
-                    P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr,
-                    P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr, sink + p * L, sink + p * k,
-                    reinterpret_cast<const int*>(sg1), k, P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr,
-                    etid);
-                sync_sel();  // every thread is done with this sigma buffer
+                const uint32_t ebar = empty_bar + 8 * buf;
+                // the sigma buffer goes back to the streamers as soon as the selector has
+                // taken its values (called after a group barrier; one arrival is expected)
+                score_and_select<kWsSelThreads>(sg0, sg1, L, k, scores_g, kept, sc, etid, sync_sel, [&] {
+                    if (etid == 0) mbar_arrive(ebar);
+                });
+                // the kept rows themselves move in the gather phase at the end of the kernel;
+                // here only their source positions are recorded: in idx_out when the caller
+                // wants it, else in the first word of each destination row of K_out
+                {
+                    const long long o = (long long)u * P.L_R + sink + p * k;
+                    const int row0 = sink + p * L;
+                    if (P.idx_out != nullptr) {
+                        for (int j = etid; j < k; j += kWsSelThreads) P.idx_out[o + j] = row0 + kept[j];
+                    } else if (P.K_out != nullptr) {
+                        for (int j = etid; j < k; j += kWsSelThreads)
+                            *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::D) = row0 + kept[j];
+                    }
+                }
+                sync_sel();  // every thread is done with kept[]
+            } else if (etid == 0) {
+                mbar_arrive(empty_bar + 8 * buf);
             }
-            if (etid == 0) mbar_arrive(empty_bar + 8 * buf);
         }
     } else {
         // ===================================================================== copy warp
@@ -363,6 +381,58 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         if (dead) {
             const unsigned long long t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
+        }
+    }
+
+    // ================================================================== gather phase
+    // Every warp of the CTA now moves the kept rows of the CTA's own partitions.  Doing it
+    // here, with the whole CTA and many loads in flight per thread, instead of partition
+    // by partition beside the streamers, keeps the gather off the latency of a saturated
+    // memory system.
+    __syncthreads();
+    if (P.K_out != nullptr && *abort_flag == 0) {
+        constexpr int NTALL = G::NT + kWsEpiWarps * 32;
+        constexpr int U = 8;
+        const int items = k * 2 * G::VPR;  // 32 consecutive items = one kept row of K and of V
+        for (long long s = s_first; s < s_hi; ++s) {
+            const int u = int(s / n), p = n - 1 - int(s % n);
+            if (p == n - 1) continue;
+            const uint16_t* srcK = unit_base(P.K, u);
+            const uint16_t* srcV = unit_base(P.V, u);
+            const long long o = (long long)u * P.L_R + sink + p * k;
+            uint16_t* dstK = P.K_out + o * G::D;
+            uint16_t* dstV = P.V_out + o * G::D;
+            for (int base = 0; base < items; base += NTALL * U) {
+                int src[U];
+                uint4 buf[U];
+#pragma unroll
+                for (int q = 0; q < U; ++q) {
+                    const int i = base + q * NTALL + tid;
+                    if (i < items) {
+                        const int j = (i / G::VPR) >> 1;
+                        src[q] = P.idx_out != nullptr ? __ldcg(P.idx_out + o + j)
+                                                      : __ldcg(reinterpret_cast<const int32_t*>(dstK + (long long)j * G::D));
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < U; ++q) {
+                    const int i = base + q * NTALL + tid;
+                    if (i < items) {
+                        const int vec = i % G::VPR, r2 = i / G::VPR;
+                        const uint16_t* sp = (r2 & 1) ? srcV : srcK;
+                        buf[q] = ld_nc(reinterpret_cast<const uint4*>(sp + (long long)src[q] * P.ss) + vec);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < U; ++q) {
+                    const int i = base + q * NTALL + tid;
+                    if (i < items) {
+                        const int vec = i % G::VPR, r2 = i / G::VPR, j = r2 >> 1;
+                        uint16_t* dp = (r2 & 1) ? dstV : dstK;
+                        st_stream(reinterpret_cast<uint4*>(dp + (long long)j * G::D) + vec, buf[q]);
+                    }
+                }
+            }
         }
     }
 }

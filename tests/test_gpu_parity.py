@@ -211,11 +211,14 @@ def test_zero_range_channel(binding, oracle):
     check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host)
 
 
-def test_indices_only_and_rows_only(binding, oracle):
+@pytest.mark.parametrize("warps", [0, 12])
+def test_indices_only_and_rows_only(binding, oracle, warps):
     B, H, D, sink, L, k = 1, 3, 128, 8, 128, 32
     S = sink + 4 * L + 17
     K, V = synth.make_kv(B, H, S, D, seed=17, device="cuda:0")
     plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    if warps:
+        plan.tune(warps=warps, tile_rows=32, stages=2, ctas_per_sm=1)
     ws = plan.new_workspace()
     full = plan.compress_prefill(K, V, ws)
     only_idx = plan.compress_prefill(K, V, ws, want_rows=False)
