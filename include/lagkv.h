@@ -49,7 +49,8 @@ enum lagkv_status {
     LAGKV_EWORKSPACE = 3,   /* workspace missing or too small                         */
     LAGKV_ECUDA = 4,        /* CUDA runtime error at launch (left sticky, not cleared)*/
     LAGKV_ETIMEOUT = 5,     /* device: a bounded wait on an async copy ran out        */
-    LAGKV_ECAPACITY = 6     /* device: append needed more chunks than max_new_chunks  */
+    LAGKV_ECAPACITY = 6,    /* device: append needed more chunks than max_new_chunks  */
+    LAGKV_ENOALLOC_LIMIT = 7 /* request larger than LAGKV_NOALLOC_SCRATCH_BYTES        */
 };
 
 enum lagkv_variant {
@@ -149,6 +150,44 @@ int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64
                           int32_t *seq_len, int32_t *static_len, int32_t max_new_chunks,
                           int32_t *idx_out, float *scores_out, void *workspace,
                           size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * lagkv_compress_append() for callers that have no device memory to give as a workspace.
+ * (The paper has no counterpart: this is a property of the library, not of the method.)
+ *
+ * Who needs it: code that runs where allocating is off the table -- a decode loop inside a
+ * serving engine whose memory pool is already carved up, a plug-in called from someone
+ * else's stream callback or capture region, a host that forbids cudaMalloc after start-up
+ * because it would synchronise the device.  Such a caller cannot produce the workspace
+ * that lagkv_compress_append() wants, so the library brings its own: a fixed array of
+ * LAGKV_NOALLOC_SCRATCH_BYTES bytes inside the library image.  Every GPU that loads the
+ * library holds one copy of it until the process exits.
+ *
+ * Arguments are those of lagkv_compress_append() minus workspace / workspace_bytes, plus
+ *   status_out  DEVICE int32[4] or NULL: receives the status block of this call (same
+ *               meaning as lagkv_read_status(): [0] first device-side status, [1] detail,
+ *               [2] zero-range channel count), written on cuda_stream after the kernels.
+ * The call allocates nothing and frees nothing; it enqueues a 256-byte memset, the append
+ * kernels and, if asked, a 16-byte device-to-device copy.
+ *
+ * Limit: 256 + B*H_kv*max_new_chunks*k*4 bytes must not exceed LAGKV_NOALLOC_SCRATCH_BYTES
+ * when idx_out is NULL (the kept positions are parked in the scratch); with idx_out given
+ * only the 256-byte status block is used.  Beyond the limit the call returns
+ * LAGKV_ENOALLOC_LIMIT and touches nothing.
+ *
+ * First call on a device: the library looks up the device address of its array (once per
+ * device, with that device current).  Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, and the array keeps whatever the last
+ * call left in it.  The status block is cleared at the start of every call; the kept
+ * positions are rewritten before they are read.  Two calls that overlap on the GPU (two
+ * streams, no dependency between them) race on the array: order them.
+ */
+#define LAGKV_NOALLOC_SCRATCH_BYTES 1048576
+int lagkv_compress_append_noalloc(lagkv_plan_t plan, void *K_cache, void *V_cache, int64_t S_cap,
+                                  int32_t *seq_len, int32_t *static_len, int32_t max_new_chunks,
+                                  int32_t *idx_out, float *scores_out, int32_t *status_out,
+                                  void *cuda_stream);
 
 /*
  * Row gather, the separable part of the compaction (Fig. 1):

@@ -19,13 +19,16 @@ import torch
 LIB_PATH = Path(__file__).resolve().parent / "liblagkv_b200.so"
 
 LAGKV_OK, LAGKV_EINVAL, LAGKV_EUNSUPPORTED, LAGKV_EWORKSPACE, LAGKV_ECUDA, LAGKV_ETIMEOUT, LAGKV_ECAPACITY = range(7)
+LAGKV_ENOALLOC_LIMIT = 7
+NOALLOC_SCRATCH_BYTES = 1048576
 VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
 
 # every symbol include/lagkv.h declares
 EXPORTS = (
     "lagkv_plan", "lagkv_plan_destroy", "lagkv_keep_count", "lagkv_compressed_len",
     "lagkv_keep_for_target", "lagkv_workspace_bytes", "lagkv_workspace_init",
-    "lagkv_compress_prefill", "lagkv_compress_append", "lagkv_gather", "lagkv_read_status",
+    "lagkv_compress_prefill", "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
+    "lagkv_read_status",
     "lagkv_launch_info", "lagkv_plan_tune", "lagkv_status_string", "lagkv_version",
 )
 
@@ -79,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_compress_prefill.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
     lib.lagkv_compress_append.restype = ctypes.c_int
     lib.lagkv_compress_append.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.lagkv_compress_append_noalloc.restype = ctypes.c_int
+    lib.lagkv_compress_append_noalloc.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.lagkv_gather.restype = ctypes.c_int
     lib.lagkv_gather.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
     lib.lagkv_read_status.restype = ctypes.c_int
@@ -227,6 +232,23 @@ class Plan:
             int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(workspace), workspace.numel(), _stream(dev))
         _check(rc, "lagkv_compress_append")
 
+    def compress_append_noalloc(self, K_cache, V_cache, seq_len, static_len, max_new_chunks=1, idx_out=None,
+                                scores_out=None, status_out=None):
+        """``lagkv_compress_append_noalloc``: the append pass for callers that cannot hand over a
+        workspace.  The library's own fixed scratch array is used instead; nothing is
+        allocated here either (every tensor, ``status_out`` int32[4] included, is the
+        caller's).  Raises ``LagKVError`` with ``LAGKV_ENOALLOC_LIMIT`` when the kept-position
+        list would not fit the built-in array."""
+        self._check_cache(K_cache, "K_cache")
+        self._check_cache(V_cache, "V_cache")
+        for t, name in ((seq_len, "seq_len"), (static_len, "static_len")):
+            if t.dtype != torch.int32 or not t.is_cuda or t.numel() != self.cfg.B or not t.is_contiguous():
+                raise TypeError(f"{name} must be a contiguous int32 CUDA tensor [B]")
+        rc = self.lib.lagkv_compress_append_noalloc(
+            self.handle, _ptr(K_cache), _ptr(V_cache), int(K_cache.shape[2]), _ptr(seq_len), _ptr(static_len),
+            int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(status_out), _stream(self._dev()))
+        _check(rc, "lagkv_compress_append_noalloc")
+
     def gather(self, K, V, idx, workspace=None, S_in=None):
         """``lagkv_gather``: rows ``idx`` ``[B, H, n_idx]`` int32 of K (and V, may be None)."""
         self._check_cache(K, "K")
@@ -259,6 +281,10 @@ def lagkv_compress_prefill(plan: Plan, K, V, workspace, **kw):
 
 def lagkv_compress_append(plan: Plan, K_cache, V_cache, seq_len, static_len, workspace, **kw):
     return plan.compress_append(K_cache, V_cache, seq_len, static_len, workspace, **kw)
+
+
+def lagkv_compress_append_noalloc(plan: Plan, K_cache, V_cache, seq_len, static_len, **kw):
+    return plan.compress_append_noalloc(K_cache, V_cache, seq_len, static_len, **kw)
 
 
 def lagkv_gather(plan: Plan, K, V, idx, **kw):

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "lagkv_kernels.cuh"
@@ -470,6 +471,7 @@ const char* lagkv_status_string(int status) {
         case LAGKV_ECUDA: return "CUDA error";
         case LAGKV_ETIMEOUT: return "device wait timed out";
         case LAGKV_ECAPACITY: return "append needs more chunks than max_new_chunks";
+        case LAGKV_ENOALLOC_LIMIT: return "request exceeds the library's built-in scratch (LAGKV_NOALLOC_SCRATCH_BYTES)";
         default: return "unknown status";
     }
 }
@@ -477,3 +479,53 @@ const char* lagkv_status_string(int status) {
 const char* lagkv_version(void) { return "lagkv-b200 0.1 (sm_100a)"; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ append without a workspace
+// Scratch that lagkv_compress_append_noalloc() hands to the append kernel in place of a
+// caller-supplied workspace: the 256-byte status block followed by the kept-position list.
+// It lives in the library image, one copy per GPU that loads the library, until the process
+// exits.  In host code the symbol below is only a handle: the address a kernel can use comes
+// from cudaGetSymbolAddress(), asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LAGKV_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device` (which must be current); nullptr on error.
+void* noalloc_scratch_for(int device) {
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[device] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
+        g_noalloc_ptr[device] = ptr;
+    }
+    return g_noalloc_ptr[device];
+}
+}  // namespace
+
+extern "C" int lagkv_compress_append_noalloc(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap,
+                                             int32_t* seq_len, int32_t* static_len, int32_t max_new_chunks,
+                                             int32_t* idx_out, float* scores_out, int32_t* status_out,
+                                             void* cuda_stream) {
+    if (plan == nullptr || plan->cfg.device < 0 || max_new_chunks < 1) return LAGKV_EINVAL;
+    if (reinterpret_cast<uintptr_t>(status_out) & 3u) return LAGKV_EINVAL;
+    // without idx_out the kernel parks the kept positions in the scratch: that list must fit
+    const size_t need = idx_out ? kStatusWords * sizeof(int32_t) : lagkv_workspace_bytes(plan, max_new_chunks);
+    if (need == 0 || need > size_t(LAGKV_NOALLOC_SCRATCH_BYTES)) return LAGKV_ENOALLOC_LIMIT;
+    DeviceGuard guard(plan->cfg.device);
+    void* scratch = noalloc_scratch_for(plan->cfg.device);
+    if (scratch == nullptr) return LAGKV_ECUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps what the previous call left: the status block has to start at zero
+    if (cudaMemsetAsync(scratch, 0, kStatusWords * sizeof(int32_t), stream) != cudaSuccess) return LAGKV_ECUDA;
+    const int rc = lagkv_compress_append(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out,
+                                         scores_out, scratch, size_t(LAGKV_NOALLOC_SCRATCH_BYTES), stream);
+    if (rc != LAGKV_OK) return rc;
+    if (status_out != nullptr &&
+        cudaMemcpyAsync(status_out, scratch, 4 * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return LAGKV_ECUDA;
+    return LAGKV_OK;
+}
