@@ -1,0 +1,130 @@
+"""GPU parity at the full sizes of the benchmark configurations, in the launch configuration
+``bench.py`` times (layers folded into the batch, planner defaults): properties that hold at any
+size over the whole result, plus randomly sampled partitions recomputed one by one by the
+float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as pu
+from paper_2504_04704_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2504_04704_b200 import binding as b
+    b.load_library()
+    return b
+
+
+def folded_cache(w, dev="cuda:0"):
+    Bf = w.layers * w.B
+    K = torch.empty((Bf, w.H, w.S, w.D), dtype=torch.bfloat16, device=dev)
+    V = torch.empty_like(K)
+    for layer in range(w.layers):
+        K[layer * w.B:(layer + 1) * w.B], V[layer * w.B:(layer + 1) * w.B] = synth.make_workload_layer(w, layer, device=dev)
+    return K, V
+
+
+@pytest.mark.parametrize("name,samples", [("llama8b_32k", 48), ("llama8b_128k", 48)])
+def test_full_size_prefill(binding, oracle, name, samples):
+    w = synth.WORKLOADS[name]
+    K, V = folded_cache(w)
+    plan = binding.Plan(w.layers * w.B, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, device=0)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill(K, V, ws, want_scores=True)
+    st = plan.read_status(ws)
+    assert st[0] == 0, st
+    assert out["L_R"] == {"llama8b_32k": 9728, "llama8b_128k": 19968}[name]
+    pu.check_structure(K, V, out, w.sink, w.lag, plan.k, w.S, chunk_units=32)
+    exact, total = pu.check_samples(oracle, K, V, out, w.sink, w.lag, plan.k, w.S, samples, seed=7)
+    print(f"{name}: {exact}/{total} sampled partitions identical to the oracle, the rest explained near-ties; "
+          f"zero-range channels {st[2]}; launch {plan.launch_info(w.S)}")
+
+
+CELLS = [(L, r) for L in (64, 128, 256, 512, 1024, 2048) for r in (0.5, 0.25, 0.125, 0.0625)]
+
+
+@pytest.mark.parametrize("B", [1, 8])
+def test_full_size_sweep(binding, oracle, B):
+    """Config 4: Ls = 65536, sink = 4, every (L, r) cell, seed per cell."""
+    w = synth.WORKLOADS["sweep"]
+    mism = 0
+    for cell, (L, r) in enumerate(CELLS):
+        K, V = synth.make_kv(B, w.H, w.S, w.D, seed=4000 + 100 * cell + B, device="cuda:0")
+        plan = binding.Plan(B, w.H, w.D, w.sink, L, keep_ratio=r, device=0)
+        assert plan.k == int(round(r * L))
+        ws = plan.new_workspace()
+        out = plan.compress_prefill(K, V, ws, want_scores=True)
+        assert plan.read_status(ws)[0] == 0
+        pu.check_structure(K, V, out, w.sink, L, plan.k, w.S)
+        exact, total = pu.check_samples(oracle, K, V, out, w.sink, L, plan.k, w.S, 6, seed=cell)
+        mism += total - exact
+        del K, V, out
+    print(f"sweep B={B}: {mism} sampled partitions differed from the oracle by explained near-ties")
+
+
+def test_full_size_decode_append(binding, oracle):
+    """Config 3: B = 16 sequences x 28 layers folded, 4 KV heads, L = 512, k = 128.  Every
+    sequence starts with 16384 stored rows (16 sink + 123 x 128 kept + 624 window) and grows
+    by 4096 tokens; the append entry point is called after every block of new tokens, which
+    triggers 8 compressions of one partition each (after 400, 912, ... appended tokens) and
+    skips otherwise.  Sampled sequences are replayed by the oracle."""
+    w = synth.WORKLOADS["decode_append"]
+    Bf, H, D, L, sink = w.layers * w.B, w.H, w.D, w.lag, w.sink
+    plan = binding.Plan(Bf, H, D, sink, L, keep_ratio=w.ratio, device=0)
+    k = plan.k
+    start, grow = 16384, 4096
+    S_cap = start + 8 * k + 2 * L            # the stored cache grows by k rows per trigger
+    stat0 = sink + 123 * k
+    assert start - stat0 == L + 112
+    K = torch.empty((Bf, H, S_cap, D), dtype=torch.bfloat16, device="cuda:0")
+    V = torch.empty_like(K)
+    Knew = torch.empty((Bf, H, grow, D), dtype=torch.bfloat16, device="cuda:0")
+    Vnew = torch.empty_like(Knew)
+    for layer in range(w.layers):
+        sl = slice(layer * w.B, (layer + 1) * w.B)
+        k_l, v_l = synth.make_kv(w.B, H, start + grow, D, w.seed(layer), device="cuda:0")
+        K[sl, :, :start], V[sl, :, :start] = k_l[:, :, :start], v_l[:, :, :start]
+        Knew[sl], Vnew[sl] = k_l[:, :, start:], v_l[:, :, start:]
+    seq = torch.full((Bf,), start, dtype=torch.int32, device="cuda:0")
+    stat = torch.full((Bf,), stat0, dtype=torch.int32, device="cuda:0")
+    ws = plan.new_workspace(1)
+    rng = np.random.default_rng(3)
+    sample = sorted({0, Bf - 1, *map(int, rng.integers(Bf, size=4))})
+    ref = {b: (synth.to_bits(K[b:b + 1]), synth.to_bits(V[b:b + 1]), np.array([start]), np.array([stat0])) for b in sample}
+
+    done, triggers, calls = 0, 0, 0
+    blocks = [200, 200] + [256, 256] * 8          # 400, then 512 per trigger; ends at 4496 > 4096: clipped
+    for step in blocks:
+        step = min(step, grow - done)
+        if step == 0:
+            break
+        cur = int(seq[0])                          # all sequences advance together in this workload
+        K[:, :, cur:cur + step], V[:, :, cur:cur + step] = Knew[:, :, done:done + step], Vnew[:, :, done:done + step]
+        seq += step
+        before = int(stat[0])
+        plan.compress_append(K, V, seq, stat, ws, max_new_chunks=1)
+        calls += 1
+        triggers += int(stat[0]) != before
+        for b in sample:
+            Kb, Vb, sb, tb = ref[b]
+            c = int(sb[0])
+            Kb[:, :, c:c + step] = synth.to_bits(Knew[b:b + 1, :, done:done + step])
+            Vb[:, :, c:c + step] = synth.to_bits(Vnew[b:b + 1, :, done:done + step])
+            Kb, Vb, sb, tb, _ = oracle.compress_append(Kb, Vb, sb + step, tb, L, k)
+            ref[b] = (Kb, Vb, sb, tb)
+        done += step
+    assert plan.read_status(ws)[0] == 0
+    assert done == grow and triggers == 8
+    assert seq.tolist() == [stat0 + 8 * k + L + (start - stat0 - L + grow) % L] * Bf
+    assert stat.tolist() == [stat0 + 8 * k] * Bf
+    for b in sample:
+        Kb, Vb, sb, tb = ref[b]
+        m = int(sb[0])
+        assert int(seq[b]) == m and int(stat[b]) == int(tb[0])
+        np.testing.assert_array_equal(synth.to_bits(K[b:b + 1, :, :m]), Kb[:, :, :m])
+        np.testing.assert_array_equal(synth.to_bits(V[b:b + 1, :, :m]), Vb[:, :, :m])
+    print(f"decode_append: {calls} calls, {triggers} triggers, {len(sample)} sequences replayed by the oracle")
