@@ -191,7 +191,7 @@ def main():
     import torch
     import torch.distributed as dist
     import __graft_entry__
-    from paper_2504_04704_b200 import binding
+    from paper_2504_04704_b200 import binding, shard
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -210,7 +210,7 @@ def main():
     K = torch.empty((Bf, w.H, w.S, w.D), dtype=torch.bfloat16, device=dev)
     V = torch.empty_like(K)
     for layer in range(w.layers):
-        k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, w.seed(layer) + 100000 * rank, w.sigma_k, w.sigma_v, device=dev)
+        k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, shard.rank_seed(w.seed(layer), rank), w.sigma_k, w.sigma_v, device=dev)
         K[layer * w.B:(layer + 1) * w.B], V[layer * w.B:(layer + 1) * w.B] = k_l, v_l
         del k_l, v_l
     plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, device=local)
@@ -248,14 +248,11 @@ def main():
     ms_total = e0.elapsed_time(e1)
     status = plan.read_status(ws)
     assert status[0] == 0, f"device status {status}"
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = shard.max_over_ranks(ms_total, dev)
     clocks = sampler.stop(wall0, wall1) if sampler else None
     ms_step = ms_total / args.steps
     units_per_rank = w.layers * w.B * w.H * w.S
-    value = world * units_per_rank / (ms_step * 1e-3)
+    value = shard.job_throughput(units_per_rank, world, ms_step)
 
     # ---- end to end: host cache -> device -> compress -> compacted cache back on the host
     e2e = None
@@ -283,11 +280,8 @@ def main():
         f1.record(stream)
         torch.cuda.synchronize()
         ms_e2e = f0.elapsed_time(f1) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * units_per_rank / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+        ms_e2e = shard.max_over_ranks(ms_e2e, dev)
+        e2e = {"value": shard.job_throughput(units_per_rank, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": hp.h2d_bytes, "d2h_bytes_per_step": hp.d2h_bytes, "steps": args.e2e_steps,
                "chunk_layers": chunk // w.B}
         del Kh, Vh, Koh, Voh, Ih, hp

@@ -4,4 +4,4 @@
 seeded input generators.  Importing the package loads nothing native: the shared
 library is opened on the first call into ``binding`` and a missing library is an error.
 """
-__all__ = ["binding", "synth"]
+__all__ = ["binding", "synth", "shard"]
