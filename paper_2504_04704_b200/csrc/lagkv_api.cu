@@ -30,8 +30,8 @@ struct KernelEntry {
 
 #define LAGKV_ENTRY(D, V, NW, TR) \
     { D, NW, TR, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
-#define LAGKV_WS_ENTRY(D, V, TR) \
-    { D, 8 + kWsEpiWarps, TR, true, &lagkv_ws_kernel<Geo<D, V, 8, TR>>, &ws_smem_total_bytes<Geo<D, V, 8, TR>> }
+#define LAGKV_WS_ENTRY(D, V, NWS, TR) \
+    { D, NWS + kWsEpiWarps, TR, true, &lagkv_ws_kernel<Geo<D, V, NWS, TR>>, &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
 
 const KernelEntry kKernels[] = {
     LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
@@ -40,8 +40,8 @@ const KernelEntry kKernels[] = {
     LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
     LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
     LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
-    LAGKV_WS_ENTRY(128, 2, 32), LAGKV_WS_ENTRY(128, 2, 16), LAGKV_WS_ENTRY(64, 1, 32), LAGKV_WS_ENTRY(64, 1, 16),
-    LAGKV_WS_ENTRY(256, 2, 16),
+    LAGKV_WS_ENTRY(128, 2, 8, 32), LAGKV_WS_ENTRY(128, 2, 8, 16), LAGKV_WS_ENTRY(64, 1, 8, 32),
+    LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16),
 };
 constexpr int kNumKernels = int(sizeof(kKernels) / sizeof(kKernels[0]));
 

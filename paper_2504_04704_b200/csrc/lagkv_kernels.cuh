@@ -26,7 +26,7 @@
 namespace lagkv {
 
 constexpr int kStatusWords = 64;  // 256-byte status block at the start of the workspace
-constexpr int kMaxWarps = 8;
+constexpr int kMaxWarps = 16;
 
 enum { MODE_PREFILL = 0, MODE_APPEND = 1 };
 enum { ST_OK = 0, ST_EINVAL = 1, ST_ETIMEOUT = 5, ST_ECAPACITY = 6 };
@@ -306,6 +306,58 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
             sig_out[row] = sqrtf(var);
         }
     }
+}
+
+// ------------------------------------------------------------------ coefficients of Eq. 9
+// Combine the per-warp min / max partials of one tensor (nw rows of [mn | mx], STAT words
+// each, packed bf16x2) and turn them into y = a * z + b for this lane's channels:
+// y = (z - mid) / range, a shift of Eq. 9 by -1/2 that leaves the std unchanged.  A channel
+// whose range is zero gets a = 0 (y constant).  Returns how many of this lane's channels
+// had zero range.  The reciprocal is the hardware approximation (1 ulp), the same in every
+// kernel, so scores do not depend on which kernel ran.
+template <class G>
+__device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw, int cg, f32x2 (&a2)[G::NWORD],
+                                                 f32x2 (&b2)[G::NWORD]) {
+    constexpr int STAT = G::D / 2;
+    uint32_t fmn[G::NWORD], fmx[G::NWORD];
+#pragma unroll
+    for (int j = 0; j < G::NWORD; ++j) {
+        fmn[j] = 0x7f807f80u;
+        fmx[j] = 0xff80ff80u;
+    }
+    for (int w = 0; w < nw; ++w) {
+        const uint4* st = reinterpret_cast<const uint4*>(stats_t + w * 2 * STAT);
+#pragma unroll
+        for (int v = 0; v < G::V; ++v) {
+            const uint4 lo = st[v * G::LPR + cg], hi = st[STAT / 4 + v * G::LPR + cg];
+            fmn[v * 4 + 0] = bf2_min(fmn[v * 4 + 0], lo.x);
+            fmn[v * 4 + 1] = bf2_min(fmn[v * 4 + 1], lo.y);
+            fmn[v * 4 + 2] = bf2_min(fmn[v * 4 + 2], lo.z);
+            fmn[v * 4 + 3] = bf2_min(fmn[v * 4 + 3], lo.w);
+            fmx[v * 4 + 0] = bf2_max(fmx[v * 4 + 0], hi.x);
+            fmx[v * 4 + 1] = bf2_max(fmx[v * 4 + 1], hi.y);
+            fmx[v * 4 + 2] = bf2_max(fmx[v * 4 + 2], hi.z);
+            fmx[v * 4 + 3] = bf2_max(fmx[v * 4 + 3], hi.w);
+        }
+    }
+    int zero_range = 0;
+#pragma unroll
+    for (int j = 0; j < G::NWORD; ++j) {
+        const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
+        const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
+        const float r0 = hi0 - lo0, r1 = hi1 - lo1;
+        float i0, i1;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(i0) : "f"(r0));
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(i1) : "f"(r1));
+        const float a0 = r0 > 0.f ? i0 : 0.f, a1 = r1 > 0.f ? i1 : 0.f;
+        const float c0 = r0 > 0.f ? -(0.5f * (lo0 + hi0)) * a0 : -0.5f;
+        const float c1 = r1 > 0.f ? -(0.5f * (lo1 + hi1)) * a1 : -0.5f;
+        zero_range += !(r0 > 0.f);
+        zero_range += !(r1 > 0.f);
+        a2[j] = pack2(a0, a1);
+        b2[j] = pack2(c0, c1);
+    }
+    return zero_range;
 }
 
 // -------------------------------------------------------------- softmax + top-k (block)
@@ -936,39 +988,9 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
             }
         }
 
-        // ---- coefficients for the next (lower) partition from this one's statistics:
-        //      y = (z - mid) / range, a shift of Eq. 9 by -1/2 that leaves the std unchanged
+        // ---- coefficients for the next (lower) partition from this one's statistics
         {
-            uint32_t fmn[G::NWORD], fmx[G::NWORD];
-#pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
-                fmn[j] = 0x7f807f80u;
-                fmx[j] = 0xff80ff80u;
-            }
-            for (int w = 0; w < G::WT; ++w) {
-                const uint32_t* st = stats + ((tensor * G::WT + w) * 2) * (G::D / 2);
-#pragma unroll
-                for (int v = 0; v < G::V; ++v)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        fmn[v * 4 + c] = bf2_min(fmn[v * 4 + c], st[(v * G::LPR + cg) * 4 + c]);
-                        fmx[v * 4 + c] = bf2_max(fmx[v * 4 + c], st[(G::D / 2) + (v * G::LPR + cg) * 4 + c]);
-                    }
-            }
-            int zero_range = 0;
-#pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
-                const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
-                const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
-                const float r0 = hi0 - lo0, r1 = hi1 - lo1;
-                const float a0 = r0 > 0.f ? 1.0f / r0 : 0.f, a1 = r1 > 0.f ? 1.0f / r1 : 0.f;
-                const float c0 = r0 > 0.f ? -(0.5f * (lo0 + hi0)) * a0 : -0.5f;
-                const float c1 = r1 > 0.f ? -(0.5f * (lo1 + hi1)) * a1 : -0.5f;
-                zero_range += !(r0 > 0.f);
-                zero_range += !(r1 > 0.f);
-                a2[j] = pack2(a0, a1);
-                b2[j] = pack2(c0, c1);
-            }
+            const int zero_range = make_coefficients<G>(stats + (tensor * G::WT) * 2 * (G::D / 2), G::WT, cg, a2, b2);
             if (zero_range != 0 && wj == 0 && rl == 0 && P.status != nullptr) atomicAdd(P.status + 2, zero_range);
             have_ref = true;
         }

@@ -111,14 +111,17 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         bool dead = false;
 
         const bool has_tiles = wj < ntiles;
-        long long ps = s_lo;  // producer cursor: next tile to request
+        // producer cursor: next tile to request, kept as (slots left, unit, partition, tile)
+        // and advanced without divisions
+        long long pleft = s_hi - s_lo;
+        int pu = int(s_lo / n), pp = n - 1 - int(s_lo % n);
+        const uint16_t* pbase = unit_base(tbase, pu);
         int pt = wj, pslot = 0;
         auto issue_next = [&]() {  // warp-collective
-            if (dead || !has_tiles || ps >= s_hi) return;
-            const int u = int(ps / n), p = n - 1 - int(ps % n);
-            const int row0 = sink + p * L + pt * G::TR;
+            if (dead || !has_tiles || pleft <= 0) return;
+            const int row0 = sink + pp * L + pt * G::TR;
             const int rows = min(G::TR, L - pt * G::TR);
-            const uint16_t* src = unit_base(tbase, u) + (long long)row0 * P.ss;
+            const uint16_t* src = pbase + (long long)row0 * P.ss;
             const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
             const uint32_t bar = bar_w + 8 * pslot;
             const uint32_t bytes = uint32_t(rows) * G::D * 2;
@@ -134,9 +137,14 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
             }
             pt += G::WT;
-            if (pt >= ntiles) {
+            if (pt >= ntiles) {  // next slot: the partition below, or the top of the next unit
                 pt = wj;
-                ++ps;
+                --pleft;
+                if (--pp < 0) {
+                    pp = n - 1;
+                    ++pu;
+                    pbase = unit_base(tbase, pu);
+                }
             }
             if (++pslot == NS) pslot = 0;
         };
@@ -149,9 +157,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
 #pragma unroll
         for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
 
-        for (long long s = s_lo; s < s_hi; ++s) {
+        int p = n - 1 - int(s_lo % n);
+        for (long long s = s_lo; s < s_hi; ++s, p = (p == 0 ? n - 1 : p - 1)) {
             const int i = int(s - s_lo), buf = i & 1;
-            const int p = n - 1 - int(s % n);
             const bool score = (p != n - 1) && s >= s_first;
             dead = __any_sync(0xffffffffu, dead || *abort_flag != 0);
             // the select warps must have released this sigma buffer (slot i - 2)
@@ -218,39 +226,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             // sigma of this tensor is complete: hand the slot to the select warps
             if (lane == 0) mbar_arrive(full_bar + 8 * buf);
 
-            // ---- coefficients for the next (lower) partition from this one's statistics:
-            //      y = (z - mid) / range, a shift of Eq. 9 by -1/2 that leaves the std unchanged
+            // ---- coefficients for the next (lower) partition from this one's statistics
             {
-                uint32_t fmn[G::NWORD], fmx[G::NWORD];
-#pragma unroll
-                for (int j = 0; j < G::NWORD; ++j) {
-                    fmn[j] = 0x7f807f80u;
-                    fmx[j] = 0xff80ff80u;
-                }
-                for (int w = 0; w < G::WT; ++w) {
-                    const uint32_t* st = stats_t + w * 2 * STAT_WORDS;
-#pragma unroll
-                    for (int v = 0; v < G::V; ++v)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            fmn[v * 4 + c] = bf2_min(fmn[v * 4 + c], st[(v * G::LPR + cg) * 4 + c]);
-                            fmx[v * 4 + c] = bf2_max(fmx[v * 4 + c], st[STAT_WORDS + (v * G::LPR + cg) * 4 + c]);
-                        }
-                }
-                int zero_range = 0;
-#pragma unroll
-                for (int j = 0; j < G::NWORD; ++j) {
-                    const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
-                    const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
-                    const float r0 = hi0 - lo0, r1 = hi1 - lo1;
-                    const float a0 = r0 > 0.f ? 1.0f / r0 : 0.f, a1 = r1 > 0.f ? 1.0f / r1 : 0.f;
-                    const float c0 = r0 > 0.f ? -(0.5f * (lo0 + hi0)) * a0 : -0.5f;
-                    const float c1 = r1 > 0.f ? -(0.5f * (lo1 + hi1)) * a1 : -0.5f;
-                    zero_range += !(r0 > 0.f);
-                    zero_range += !(r1 > 0.f);
-                    a2[j] = pack2(a0, a1);
-                    b2[j] = pack2(c0, c1);
-                }
+                const int zero_range = make_coefficients<G>(stats_t, G::WT, cg, a2, b2);
                 if (zero_range != 0 && wj == 0 && rl == 0 && !dead && P.status != nullptr)
                     atomicAdd(P.status + 2, zero_range);
             }
