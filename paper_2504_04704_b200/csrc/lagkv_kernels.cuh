@@ -361,17 +361,24 @@ __device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw
 }
 
 // -------------------------------------------------------------- softmax + top-k (block)
-// The softmax denominators are accumulated as integers (exp value times 2^40, rounded), so
+// The softmax denominators are accumulated as integers (exp value times 2^30, rounded), so
 // they do not depend on which thread adds what: the scores, and with them the selection,
 // are a function of the sigma values alone, bit-identical for every launch shape and for
-// both implementations below.
-__device__ __forceinline__ unsigned long long fx40(float e) { return __float2ull_rn(e * 1099511627776.0f); }
-__device__ __forceinline__ float fx40_to_float(unsigned long long q) {
-    return __ull2float_rn(q) * (1.0f / 1099511627776.0f);
+// both implementations below.  exp is the hardware exponential of base 2 (relative error
+// about 2^-22) and the division by the denominator a multiplication by its reciprocal:
+// both far inside the score tolerance, and the same in every kernel.
+__device__ __forceinline__ float softmax_exp(float x, float m) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"((x - m) * 1.4426950408889634f));
+    return r;
 }
-// Eq. 11 from the two exponentials and the two softmax denominators
-__device__ __forceinline__ float combine_scores(float e0, float s0, float e1, float s1) {
-    return __fadd_rn(__fdiv_rn(e0, s0), __fdiv_rn(e1, s1));
+__device__ __forceinline__ unsigned long long fx30(float e) { return __float2uint_rn(e * 1073741824.0f); }
+__device__ __forceinline__ float fx30_to_recip(unsigned long long q) {
+    return __frcp_rn(__ull2float_rn(q) * (1.0f / 1073741824.0f));
+}
+// Eq. 11 from the two exponentials and the reciprocals of the two softmax denominators
+__device__ __forceinline__ float combine_scores(float e0, float r0, float e1, float r1) {
+    return __fmaf_rn(e0, r0, __fmul_rn(e1, r1));
 }
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
@@ -426,10 +433,10 @@ __device__ void select_in_registers(const float* sg0, const float* sg1, int L, i
     unsigned long long q0 = 0, q1 = 0;
 #pragma unroll
     for (int j = 0; j < E; ++j) {
-        x0[j] = expf(x0[j] - m0);  // exp(-inf) = 0 for the padding
-        x1[j] = expf(x1[j] - m1);
-        q0 += fx40(x0[j]);
-        q1 += fx40(x1[j]);
+        x0[j] = softmax_exp(x0[j], m0);  // exp(-inf) = 0 for the padding
+        x1[j] = softmax_exp(x1[j], m1);
+        q0 += fx30(x0[j]);
+        q1 += fx30(x1[j]);
     }
     q0 = warp_sum_u64(q0);
     q1 = warp_sum_u64(q1);
@@ -444,19 +451,40 @@ __device__ void select_in_registers(const float* sg0, const float* sg1, int L, i
         q0 += sc.redq[0][w];
         q1 += sc.redq[1][w];
     }
-    const float s0 = fx40_to_float(q0), s1 = fx40_to_float(q1);
+    const float r0 = fx30_to_recip(q0), r1 = fx30_to_recip(q1);
     // ---- Eq. 11, then the order-preserving integer image; padding gets the smallest key
     uint32_t key[E];
+    uint32_t kor = 0u, kand = 0xffffffffu;
 #pragma unroll
     for (int j = 0; j < E; ++j) {
         const int t = t_lo + j;
-        const float sco = combine_scores(x0[j], s0, x1[j], s1);
+        const float sco = combine_scores(x0[j], r0, x1[j], r1);
         key[j] = t < L ? float_key(sco) : 0u;
+        if (t < L) {
+            kor |= key[j];
+            kand &= key[j];
+        }
         if (scores_g != nullptr && t < L) scores_g[t] = sco;
     }
+    // bits on which all keys agree need no search: find the highest bit where two keys differ
+    kor = __reduce_or_sync(0xffffffffu, kor);
+    kand = __reduce_and_sync(0xffffffffu, kand);
+    if (lane == 0) {
+        sc.cnt[0][warp] = int(kor);
+        sc.cnt[1][warp] = int(kand);
+    }
+    sync();
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) {
+        kor |= uint32_t(sc.cnt[0][w]);
+        kand &= uint32_t(sc.cnt[1][w]);
+    }
+    sync();  // sc.cnt is reused by the counting rounds
+    const uint32_t diff = kor ^ kand;
+    const int top = 31 - __clz(diff);  // -1 when every key is the same
     // ---- T = key of the k-th largest score: the largest T with count(key >= T) >= k
-    uint32_t T = 0;
-    for (int bit = 31; bit >= 0; --bit) {
+    uint32_t T = top >= 0 ? (kand & ~((2u << top) - 1u)) : kand;
+    for (int bit = top; bit >= 0; --bit) {
         const uint32_t cand = T | (1u << bit);
         int c = 0;
 #pragma unroll
@@ -542,11 +570,11 @@ __device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __
     }
     unsigned long long q0 = 0, q1 = 0;
     for (int t = tid; t < L; t += NT) {
-        const float e0 = expf(sg0[t] - m0), e1 = expf(sg1[t] - m1);
+        const float e0 = softmax_exp(sg0[t], m0), e1 = softmax_exp(sg1[t], m1);
         sg0[t] = e0;
         sg1[t] = e1;
-        q0 += fx40(e0);
-        q1 += fx40(e1);
+        q0 += fx30(e0);
+        q1 += fx30(e1);
     }
     q0 = warp_sum_u64(q0);
     q1 = warp_sum_u64(q1);
@@ -561,10 +589,10 @@ __device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __
         q0 += sc.redq[0][w];
         q1 += sc.redq[1][w];
     }
-    const float s0 = fx40_to_float(q0), s1 = fx40_to_float(q1);
+    const float r0 = fx30_to_recip(q0), r1 = fx30_to_recip(q1);
     // ---- Eq. 11
     for (int t = tid; t < L; t += NT) {
-        const float sco = combine_scores(sg0[t], s0, sg1[t], s1);
+        const float sco = combine_scores(sg0[t], r0, sg1[t], r1);
         sg0[t] = sco;
         if (scores_g != nullptr) scores_g[t] = sco;
     }
@@ -663,7 +691,8 @@ template <int NT, class Sync, class Release>
 __device__ __forceinline__ void score_and_select(float* sg0, float* sg1, int L, int k,
                                                  float* __restrict__ scores_g, int* kept, SelScratch& sc, int tid,
                                                  Sync sync, Release release) {
-    if (L <= NT * 8) select_in_registers<NT, 8>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    if (L <= NT * 6) select_in_registers<NT, 6>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    else if (L <= NT * 11) select_in_registers<NT, 11>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
     else if (L <= NT * 22) select_in_registers<NT, 22>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
     else select_in_shared<NT>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
 }
