@@ -213,6 +213,8 @@ struct SelScratch {
     int wsum[kMaxWarps];
     int bin;
     int krem;
+    int sel_done;  // warp-specialised kernel: slots whose kept positions are published
+    int claimed;   // warp-specialised kernel: leading slots whose kept rows the copy warp moves
     int abort;  // set by a warp whose bounded wait ran out; the CTA stops at the next barrier
 };
 
@@ -497,6 +499,7 @@ __device__ void select_in_registers(const float* sg0, const float* sg1, int L, i
 #pragma unroll
         for (int w = 0; w < NWARP; ++w) tot += sc.cnt[par][w];
         if (tot >= k) T = cand;
+        if (tot == k) break;  // exactly the k largest lie at or above T: the low bits are free
     }
     // ---- positions: tokens above T all stay; of those equal to T the first krem
     int cgt = 0, ceq = 0;

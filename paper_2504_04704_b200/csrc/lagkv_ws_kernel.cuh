@@ -12,12 +12,13 @@
 //   * 3 select warps: softmax over the partition, K + V (Eq. 11) and top-k with ties to
 //     the lower index -- one partition behind the streamers, overlapped with them.  They
 //     record where the kept rows come from; the rows move in the gather phase below.
-//   * 1 copy warp: the rows that are kept verbatim (sink and sliding window) of ALL
-//     units are cut into chunks dealt round-robin to the CTAs; the warp moves its chunks
-//     global -> shared -> global with bulk async copies, independent of the slot walk.
+//   * 1 copy warp: moves rows global -> shared -> global with bulk async copies: the kept
+//     rows of partitions whose positions are published (bandwidth the streamers leave
+//     unused), and the rows that are kept verbatim (sink and sliding window) of ALL units,
+//     cut into chunks dealt round-robin to the CTAs.
 //
-// When a CTA has walked all its slots, all of its warps together copy the kept rows of its
-// partitions to the output (gather phase).
+// When a CTA has walked all its slots, all of its warps together copy the kept rows the
+// copy warp has not claimed (gather phase).
 //
 // Every wait on an mbarrier is bounded; a warp whose wait ran out raises the CTA's abort
 // flag, records LAGKV_ETIMEOUT and from then on only keeps the barrier protocol alive so
@@ -85,6 +86,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             mbar_init(copy_bar + 8 * b, 1);
         }
         sc.abort = 0;
+        sc.sel_done = 0;
+        sc.claimed = 0;
     }
     fence_mbar_init();
     fence_proxy_async();
@@ -275,32 +278,78 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                             *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::D) = row0 + kept[j];
                     }
                 }
-                sync_sel();  // every thread is done with kept[]
+                __threadfence_block();  // the positions above are visible before the count below
+                sync_sel();             // every thread is done with kept[] and has written its share
             } else if (etid == 0) {
                 mbar_arrive(empty_bar + 8 * buf);
             }
+            if (etid == 0) *reinterpret_cast<volatile int*>(&sc.sel_done) = i + 1;  // slot i is published
         }
     } else {
         // ===================================================================== copy warp
-        // Chunks of the verbatim rows of every unit: first the window chunks, then the sink
-        // chunks of unit 0, then unit 1, ...; chunk g is handled by CTA g mod gridDim.x.
+        // Two kinds of 32-row chunks go through the same two-stage pipeline (bulk loads into
+        // shared memory, one bulk store per tensor out of it):
+        //   * gather chunks: kept rows of this CTA's partitions, as soon as the select warps
+        //     have published their positions (row by row loads, contiguous store).  While
+        //     the streamers leave bandwidth unused this moves most kept rows for free;
+        //     what is not claimed when the last slot is published is left to the gather
+        //     phase of the whole CTA;
+        //   * verbatim chunks: sink and window rows of ALL units, dealt round-robin over the
+        //     CTAs (chunk g belongs to CTA g mod gridDim.x): per unit first the window
+        //     chunks, then the sink chunks.
         const int win_rows = L + P.rem;
         const int cw = (win_rows + kWsCopyRows - 1) / kWsCopyRows, cs = (sink + kWsCopyRows - 1) / kWsCopyRows;
         const long long U = (long long)P.B * P.H;
         const long long total_chunks = U * (cw + cs);
         const bool rows_wanted = P.K_out != nullptr;
         const uint32_t stage_u32 = smem_u32(stage);
-        int pu = 0, pdst = 0, pnr = 0;  // chunk loaded in the previous round, not yet stored
+        const int nslots = int(s_hi - s_lo);
+        volatile int* sel_done = reinterpret_cast<volatile int*>(&sc.sel_done);
+        long long vg = blockIdx.x;          // next verbatim chunk of this CTA
+        int gslot = 0, gbatch = 0;          // gather cursor: slot index, batch inside it
+        bool gclaimed = false;
+        int nload = 0;                      // chunks loaded so far (stage = nload & 1)
         bool pending = false, dead = false;
-        int round = 0;
-        for (long long g = blockIdx.x;; g += gridDim.x, ++round) {
-            const bool have = g < total_chunks;
-            if (!have && !pending) break;
-            const int st = round & 1;
-            int u = 0, src = 0, dst = 0, nr = 0;
-            if (have) {
-                u = int(g / (cw + cs));
-                const int j = int(g % (cw + cs));
+        long long po = 0;                   // pending chunk: first destination row (global row index)
+        int pnr = 0;
+        for (;;) {
+            if (__any_sync(0xffffffffu, *abort_flag != 0)) dead = true;
+            // ---- pick the next chunk: a gather chunk if one is ready, else a verbatim chunk
+            int kind = 0;  // 0 none, 1 verbatim, 2 gather
+            int u = 0, src = 0, nr = 0;
+            long long o = 0;  // first destination row: u * L_R + row
+            const int done = *sel_done;
+            if (rows_wanted && !dead) {
+                if (!gclaimed) {
+                    // slots without kept rows (top partitions, the statistics-only extra slot)
+                    while (gslot < nslots) {
+                        const long long sl = s_lo + gslot;
+                        if (int(sl % n) != 0 && sl >= s_first) break;
+                        ++gslot;
+                    }
+                    if (gslot < done && done < nslots) {
+                        gclaimed = true;
+                        gbatch = 0;
+                        if (lane == 0) *reinterpret_cast<volatile int*>(&sc.claimed) = gslot + 1;
+                    }
+                }
+                if (gclaimed) {
+                    const long long sl = s_lo + gslot;
+                    const int p = n - 1 - int(sl % n);
+                    u = int(sl / n);
+                    nr = min(kWsCopyRows, k - gbatch * kWsCopyRows);
+                    o = (long long)u * P.L_R + sink + p * k + gbatch * kWsCopyRows;
+                    kind = 2;
+                    if ((++gbatch) * kWsCopyRows >= k) {
+                        gclaimed = false;
+                        ++gslot;
+                    }
+                }
+            }
+            if (kind == 0 && vg < total_chunks && !dead) {
+                u = int(vg / (cw + cs));
+                const int j = int(vg % (cw + cs));
+                int dst;
                 if (j < cw) {
                     src = sink + (n - 1) * L + j * kWsCopyRows;
                     dst = sink + (n - 1) * k + j * kWsCopyRows;
@@ -309,51 +358,65 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     src = dst = (j - cw) * kWsCopyRows;
                     nr = min(kWsCopyRows, sink - (j - cw) * kWsCopyRows);
                 }
+                o = (long long)u * P.L_R + dst;
                 if (P.idx_out != nullptr)
-                    for (int r = lane; r < nr; r += 32) P.idx_out[(long long)u * P.L_R + dst + r] = src + r;
+                    for (int r = lane; r < nr; r += 32) P.idx_out[o + r] = src + r;
+                kind = 1;
+                vg += gridDim.x;
             }
-            if (rows_wanted && !dead) {
-                if (have) {
-                    // stage `st` was last read by the store committed two rounds ago
+            const bool more = !dead && (vg < total_chunks || (rows_wanted && done < nslots));
+            if (kind == 0 && !pending) {
+                if (!more) break;
+                __nanosleep(500);  // nothing to do right now: the select warps are still at work
+                continue;
+            }
+            const bool load = kind != 0 && rows_wanted;
+            if (load) {
+                const int st = nload & 1;
+                // this stage was last read by the store committed two loads ago
+                if (lane == 0) {
+                    bulk_wait_read_all();
+                    fence_proxy_async();
+                    mbar_arrive_expect_tx(copy_bar + 8 * st, uint32_t(2 * nr) * G::D * 2);
+                }
+                __syncwarp();
+                const uint32_t dK = stage_u32 + uint32_t(2 * st) * CHUNK_BYTES, dV = dK + CHUNK_BYTES;
+                const uint16_t* bK = unit_base(P.K, u);
+                const uint16_t* bV = unit_base(P.V, u);
+                if (kind == 1 && contiguous) {
                     if (lane == 0) {
-                        bulk_wait_read_all();
-                        fence_proxy_async();
-                        mbar_arrive_expect_tx(copy_bar + 8 * st, uint32_t(2 * nr) * G::D * 2);
+                        bulk_g2s(dK, bK + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                        bulk_g2s(dV, bV + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
                     }
-                    __syncwarp();
-                    const uint32_t dK = stage_u32 + uint32_t(2 * st) * CHUNK_BYTES, dV = dK + CHUNK_BYTES;
-                    const uint16_t* sK = unit_base(P.K, u) + (long long)src * P.ss;
-                    const uint16_t* sV = unit_base(P.V, u) + (long long)src * P.ss;
-                    if (contiguous) {
-                        if (lane == 0) {
-                            bulk_g2s(dK, sK, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
-                            bulk_g2s(dV, sV, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
-                        }
-                    } else {
-                        for (int r = lane; r < nr; r += 32) {
-                            bulk_g2s(dK + uint32_t(r) * G::D * 2, sK + (long long)r * P.ss, G::D * 2, copy_bar + 8 * st);
-                            bulk_g2s(dV + uint32_t(r) * G::D * 2, sV + (long long)r * P.ss, G::D * 2, copy_bar + 8 * st);
-                        }
+                } else if (lane < nr) {  // one row of K and of V per lane
+                    int row = src + lane;
+                    if (kind == 2) {
+                        __threadfence_block();
+                        row = P.idx_out != nullptr ? __ldcg(P.idx_out + o + lane)
+                                                   : __ldcg(reinterpret_cast<const int32_t*>(P.K_out + (o + lane) * G::D));
                     }
-                }
-                if (pending) {  // the chunk loaded one round ago goes out
-                    const int pst = (round - 1) & 1;
-                    if (!mbar_wait_bounded(copy_bar + 8 * pst, uint32_t((round - 1) >> 1) & 1u)) {
-                        dead = true;
-                        raise_abort();
-                    } else if (lane == 0) {
-                        fence_proxy_async();
-                        const uint32_t sK = stage_u32 + uint32_t(2 * pst) * CHUNK_BYTES, sV = sK + CHUNK_BYTES;
-                        bulk_s2g(P.K_out + ((long long)pu * P.L_R + pdst) * G::D, sK, uint32_t(pnr) * G::D * 2);
-                        bulk_s2g(P.V_out + ((long long)pu * P.L_R + pdst) * G::D, sV, uint32_t(pnr) * G::D * 2);
-                        bulk_commit();
-                    }
+                    bulk_g2s(dK + uint32_t(lane) * G::D * 2, bK + (long long)row * P.ss, G::D * 2, copy_bar + 8 * st);
+                    bulk_g2s(dV + uint32_t(lane) * G::D * 2, bV + (long long)row * P.ss, G::D * 2, copy_bar + 8 * st);
                 }
             }
-            pending = have;
-            pu = u;
-            pdst = dst;
+            if (pending) {  // the chunk loaded before this one goes out
+                const int pl = nload - 1;  // nload still names the chunk loaded above, if any
+                const int pst = pl & 1;
+                if (!mbar_wait_bounded(copy_bar + 8 * pst, uint32_t(pl >> 1) & 1u)) {
+                    dead = true;
+                    raise_abort();
+                } else if (lane == 0) {
+                    fence_proxy_async();
+                    const uint32_t sK = stage_u32 + uint32_t(2 * pst) * CHUNK_BYTES, sV = sK + CHUNK_BYTES;
+                    bulk_s2g(P.K_out + po * G::D, sK, uint32_t(pnr) * G::D * 2);
+                    bulk_s2g(P.V_out + po * G::D, sV, uint32_t(pnr) * G::D * 2);
+                    bulk_commit();
+                }
+            }
+            pending = load;
+            po = o;
             pnr = nr;
+            if (load) ++nload;
         }
         if (lane == 0) bulk_wait_read_all();
         if (dead) {
@@ -372,7 +435,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         constexpr int NTALL = G::NT + kWsEpiWarps * 32;
         constexpr int U = 8;
         const int items = k * 2 * G::VPR;  // 32 consecutive items = one kept row of K and of V
-        for (long long s = s_first; s < s_hi; ++s) {
+        // slots the copy warp claimed are done; the rest (at least the last one) is moved here
+        const long long s_from = s_lo + *reinterpret_cast<volatile int*>(&sc.claimed);
+        for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
             const int u = int(s / n), p = n - 1 - int(s % n);
             if (p == n - 1) continue;
             const uint16_t* srcK = unit_base(P.K, u);
