@@ -148,12 +148,14 @@ int choose_shape(lagkv_plan_s* pl) {
     int rc = first_fit(pl, uni, nu, &pl->app);
     if (rc != LAGKV_OK) return rc;
     pl->pre = pl->app;
-    if (L >= 256) {
+    const bool needs_ws = pl->cfg.variant != LAGKV_VARIANT_LAGKV;  // only that kernel knows the variants
+    if (L >= 128 || needs_ws) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
         Shape sh;
         rc = first_fit(pl, ws, 3, &sh);
         if (rc == LAGKV_ECUDA) return rc;
         if (rc == LAGKV_OK) pl->pre = sh;
+        else if (needs_ws) return LAGKV_EUNSUPPORTED;
     }
     return LAGKV_OK;
 }
@@ -190,7 +192,7 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
     if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
-    if (cfg->variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
+    if (cfg->variant == LAGKV_VARIANT_L2NORM) return LAGKV_EUNSUPPORTED;
     if (cfg->D != 64 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
     if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
 
@@ -316,7 +318,8 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     P.n = int(rest / c.lag);
     P.rem = int(rest % c.lag);
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
-    P.total_slots = U * P.n;
+    P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : P.n;
+    P.total_slots = U * P.spu;
     P.stages = plan->pre.stages;
 
     const KernelEntry& ke = kKernels[plan->pre.kidx];
@@ -336,6 +339,7 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
         plan->cfg.device < 0)
         return LAGKV_EINVAL;
     if (S_cap < 1 || S_cap > 0x7fffffffll - 65536 || max_new_chunks < 1) return LAGKV_EINVAL;
+    if (plan->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;  // variants: prefill only
     if (!aligned16(K_cache) || !aligned16(V_cache) || K_cache == V_cache) return LAGKV_EINVAL;
     if ((reinterpret_cast<uintptr_t>(idx_out) & 3u) || (reinterpret_cast<uintptr_t>(scores_out) & 3u) ||
         (reinterpret_cast<uintptr_t>(seq_len) & 3u) || (reinterpret_cast<uintptr_t>(static_len) & 3u))
@@ -440,7 +444,8 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
         return LAGKV_OK;
     }
     long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
-    const long long slots = U * (rest / c.lag);
+    const long long nparts = rest / c.lag;
+    const long long slots = U * (c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (nparts - 1) : nparts);
     info[0] = int(grid < slots ? grid : slots);
     info[1] = kKernels[plan->pre.kidx].NW * 32;
     info[2] = int(plan->pre.smem);
@@ -457,6 +462,7 @@ int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t
                               stages ? stages : plan->pre.stages, ctas_per_sm ? ctas_per_sm : plan->pre.ctas_per_sm,
                               &sh);
     if (rc != LAGKV_OK) return rc;
+    if (!kKernels[sh.kidx].ws && plan->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
     plan->pre = sh;
     if (!kKernels[sh.kidx].ws) plan->app = sh;
     return LAGKV_OK;

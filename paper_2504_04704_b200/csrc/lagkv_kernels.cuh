@@ -46,6 +46,7 @@ struct Params {
     long long total_slots;      // prefill: U * n
     int B, H, L, k, ddof, variant, mode;
     int S_in, sink, n, rem, L_R;  // prefill
+    int spu;                      // prefill, warp-specialised kernel: slots per (b, h) unit
     int max_chunks;               // append
     int stages;                   // ring depth per warp
 };

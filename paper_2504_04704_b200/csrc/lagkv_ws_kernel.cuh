@@ -73,7 +73,14 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     // re-reads the partition above it (statistics only)
     const long long s_first = P.total_slots * blockIdx.x / gridDim.x;
     const long long s_hi = P.total_slots * (blockIdx.x + 1) / gridDim.x;
-    const bool extra = s_first < s_hi && (s_first % n) != 0;
+    // Slot j of a unit.  LagKV (Eq. 7-9): partitions n-1 ... 0, each scored with the statistics
+    // of the slot before it.  LocalKV (Eq. 14, Eq. 15): partitions n-2 ... 0, each visited
+    // twice in a row, once for its own statistics and once to be scored with them.
+    const int spu = P.spu;
+    const bool local_stats = P.variant == 1;
+    auto slot_part = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : n - 1 - j; };
+    auto slot_scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : j != 0; };  // needs the slot before it
+    const bool extra = s_first < s_hi && slot_scored(int(s_first % spu));
     const long long s_lo = extra ? s_first - 1 : s_first;
 
     const uint32_t full_bar = smem_u32(xbars), empty_bar = smem_u32(xbars + 2), copy_bar = smem_u32(xbars + 4);
@@ -117,12 +124,12 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         // producer cursor: next tile to request, kept as (slots left, unit, partition, tile)
         // and advanced without divisions
         long long pleft = s_hi - s_lo;
-        int pu = int(s_lo / n), pp = n - 1 - int(s_lo % n);
+        int pu = int(s_lo / spu), pj = int(s_lo % spu);
         const uint16_t* pbase = unit_base(tbase, pu);
         int pt = wj, pslot = 0;
         auto issue_next = [&]() {  // warp-collective
             if (dead || !has_tiles || pleft <= 0) return;
-            const int row0 = sink + pp * L + pt * G::TR;
+            const int row0 = sink + slot_part(pj) * L + pt * G::TR;
             const int rows = min(G::TR, L - pt * G::TR);
             const uint16_t* src = pbase + (long long)row0 * P.ss;
             const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
@@ -140,11 +147,11 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
             }
             pt += G::WT;
-            if (pt >= ntiles) {  // next slot: the partition below, or the top of the next unit
+            if (pt >= ntiles) {  // next slot of this unit, or the first slot of the next unit
                 pt = wj;
                 --pleft;
-                if (--pp < 0) {
-                    pp = n - 1;
+                if (++pj == spu) {
+                    pj = 0;
                     ++pu;
                     pbase = unit_base(tbase, pu);
                 }
@@ -160,10 +167,10 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
 #pragma unroll
         for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
 
-        int p = n - 1 - int(s_lo % n);
-        for (long long s = s_lo; s < s_hi; ++s, p = (p == 0 ? n - 1 : p - 1)) {
+        int cj = int(s_lo % spu);
+        for (long long s = s_lo; s < s_hi; ++s, cj = (cj + 1 == spu ? 0 : cj + 1)) {
             const int i = int(s - s_lo), buf = i & 1;
-            const bool score = (p != n - 1) && s >= s_first;
+            const bool score = slot_scored(cj) && s >= s_first;
             dead = __any_sync(0xffffffffu, dead || *abort_flag != 0);
             // the select warps must have released this sigma buffer (slot i - 2)
             if (i >= 2 && !dead && !mbar_wait_bounded(empty_bar + 8 * buf, uint32_t((i >> 1) - 1) & 1u)) {
@@ -247,8 +254,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         auto sync_sel = [] { named_bar_sync(kBarSelect, kWsSelThreads); };
         for (long long s = s_lo; s < s_hi; ++s) {
             const int i = int(s - s_lo), buf = i & 1;
-            const int u = int(s / n), p = n - 1 - int(s % n);
-            const bool score = (p != n - 1) && s >= s_first;
+            const int u = int(s / spu), sj = int(s % spu), p = slot_part(sj);
+            const bool score = slot_scored(sj) && s >= s_first;
             bool bad = __any_sync(0xffffffffu, dead || *abort_flag != 0);
             if (!bad && !mbar_wait_bounded(full_bar + 8 * buf, uint32_t(i >> 1) & 1u)) {
                 bad = true;
@@ -324,7 +331,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     // slots without kept rows (top partitions, the statistics-only extra slot)
                     while (gslot < nslots) {
                         const long long sl = s_lo + gslot;
-                        if (int(sl % n) != 0 && sl >= s_first) break;
+                        if (slot_scored(int(sl % spu)) && sl >= s_first) break;
                         ++gslot;
                     }
                     if (gslot < done && done < nslots) {
@@ -335,8 +342,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 }
                 if (gclaimed) {
                     const long long sl = s_lo + gslot;
-                    const int p = n - 1 - int(sl % n);
-                    u = int(sl / n);
+                    const int p = slot_part(int(sl % spu));
+                    u = int(sl / spu);
                     nr = min(kWsCopyRows, k - gbatch * kWsCopyRows);
                     o = (long long)u * P.L_R + sink + p * k + gbatch * kWsCopyRows;
                     kind = 2;
@@ -438,8 +445,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         // slots the copy warp claimed are done; the rest (at least the last one) is moved here
         const long long s_from = s_lo + *reinterpret_cast<volatile int*>(&sc.claimed);
         for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
-            const int u = int(s / n), p = n - 1 - int(s % n);
-            if (p == n - 1) continue;
+            const int u = int(s / spu), sj = int(s % spu), p = slot_part(sj);
+            if (!slot_scored(sj)) continue;
             const uint16_t* srcK = unit_base(P.K, u);
             const uint16_t* srcV = unit_base(P.V, u);
             const long long o = (long long)u * P.L_R + sink + p * k;

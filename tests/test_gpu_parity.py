@@ -31,9 +31,9 @@ def binding():
     return b
 
 
-def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None):
+def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, variant=0):
     """Compare a GPU prefill result ``out`` (numpy arrays) with the oracle on bit patterns."""
-    ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof)
+    ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof, variant=variant)
     B, H, S, D = Kb.shape
     assert out["L_R"] == ref["L_R"]
     n_c = ref["n_c"]
@@ -83,7 +83,8 @@ def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None):
     return res
 
 
-def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=None, sigma_k=1.0, layout="bhsd"):
+def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=None, sigma_k=1.0, layout="bhsd",
+                variant=0):
     K, V = synth.make_kv(B, H, S, D, seed=seed, sigma_k=sigma_k, device="cuda:0")
     strides = (0, 0, 0)
     Kd, Vd = K, V
@@ -97,7 +98,7 @@ def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=No
         Kp[..., :D], Vp[..., :D] = K, V
         Kd, Vd = Kp, Vp
         strides = (H * S * (D + 8), S * (D + 8), D + 8)
-    plan = binding.Plan(B, H, D, sink, L, keep_k=k, std_ddof=ddof, strides=strides, device=0)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, std_ddof=ddof, strides=strides, variant=variant, device=0)
     if tune:
         plan.tune(**tune)
     ws = plan.new_workspace()
@@ -106,7 +107,7 @@ def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=No
     assert st[0] == 0, f"device status {st}"
     host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
             "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
-    return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host)
+    return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host, variant=variant)
 
 
 # ------------------------------------------------------------------------------- prefill
@@ -243,6 +244,38 @@ def test_power_of_two_channel_rescale_is_bit_invariant(binding):
     b = plan.compress_prefill(K2, V2, ws, want_scores=True)
     assert torch.equal(a["idx"], b["idx"])
     assert torch.equal(a["scores"], b["scores"])
+
+
+# ------------------------------------------------------------------------------ variants
+@pytest.mark.parametrize("L,k,S_extra,B", [(64, 16, 60, 2), (100, 25, 7, 2), (256, 1, 255, 2), (512, 128, 3, 2),
+                                           (1024, 256, 1008, 9), (2048, 256, 100, 1), (37, 5, 36, 2), (2, 1, 1, 2)])
+def test_localkv_prefill(binding, oracle, L, k, S_extra, B):
+    """LocalKV (Eq. 14, Eq. 15): min / max come from the partition that is being scored."""
+    n = 5 if L >= 512 else 9
+    run_prefill(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 7, variant=binding.VARIANT_LOCALKV)
+
+
+def test_localkv_many_units_and_minimal(binding, oracle):
+    run_prefill(binding, oracle, 37, 5, 128, 3 + 6 * 64 + 5, 3, 64, 16, seed=78, variant=binding.VARIANT_LOCALKV)
+    run_prefill(binding, oracle, 1, 2, 128, 2 * 128, 0, 128, 32, seed=10, variant=binding.VARIANT_LOCALKV)   # n = 2
+    run_prefill(binding, oracle, 2, 4, 128, 40 + 4 * 300 + 111, 40, 300, 75, seed=4, layout="padded",
+                variant=binding.VARIANT_LOCALKV)
+
+
+def test_variants_not_built_are_refused(binding):
+    with pytest.raises(binding.LagKVError) as e:
+        binding.Plan(1, 2, 128, 4, 64, variant=binding.VARIANT_L2NORM, device=0)
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+    plan = binding.Plan(1, 2, 128, 4, 64, keep_k=16, variant=binding.VARIANT_LOCALKV, device=0)
+    K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
+    seq = torch.tensor([300], dtype=torch.int32, device="cuda:0")
+    stat = torch.tensor([4], dtype=torch.int32, device="cuda:0")
+    with pytest.raises(binding.LagKVError) as e:
+        plan.compress_append(K, V, seq, stat, plan.new_workspace(4), max_new_chunks=4)
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+    with pytest.raises(binding.LagKVError) as e:
+        plan.tune(warps=2, tile_rows=16, stages=2, ctas_per_sm=1)     # the uniform kernel has no variants
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
 
 
 # -------------------------------------------------------------------------------- gather
