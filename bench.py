@@ -37,10 +37,14 @@ DEFAULT_WORKLOAD = "llama8b_128k"
 NCU_TRAFFIC_BYTES = {"llama8b_128k": 21.5e9}
 
 
-def algorithmic_bytes(w, L_R: int) -> int:
-    """Every input row read once, every output row written once, index list written once."""
+def algorithmic_bytes(w, L_R: int, variant: int = 0) -> int:
+    """Every input row read once, every output row written once, index list written once.
+    The L2-norm variant scores from K alone: of V only the L_R output rows are read."""
     units = w.layers * w.B * w.H
-    return units * ((w.S + L_R) * 2 * w.D * 2 + 4 * L_R)
+    row = w.D * 2
+    if variant == 2:
+        return units * (w.S * row + L_R * row + L_R * 2 * row + 4 * L_R)
+    return units * ((w.S + L_R) * 2 * row + 4 * L_R)
 
 
 def measured_peak():
@@ -175,6 +179,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a smaller case)")
     ap.add_argument("--tune", default="", help="warps,tile_rows,stages,ctas_per_sm override")
+    ap.add_argument("--variant", default="lagkv", choices=["lagkv", "localkv", "l2norm"],
+                    help="scoring variant of Section 4.3 (the headline metric is lagkv)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -213,7 +219,8 @@ def main():
         k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, shard.rank_seed(w.seed(layer), rank), w.sigma_k, w.sigma_v, device=dev)
         K[layer * w.B:(layer + 1) * w.B], V[layer * w.B:(layer + 1) * w.B] = k_l, v_l
         del k_l, v_l
-    plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, device=local)
+    variant = {"lagkv": 0, "localkv": 1, "l2norm": 2}[args.variant]
+    plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, variant=variant, device=local)
     if args.tune:
         t = [int(x) for x in args.tune.split(",")]
         plan.tune(warps=t[0], tile_rows=t[1], stages=t[2], ctas_per_sm=t[3])
@@ -256,7 +263,7 @@ def main():
 
     # ---- end to end: host cache -> device -> compress -> compacted cache back on the host
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and variant == 0:
         chunk = max(1, min(4, w.layers)) * w.B
         while Bf % chunk:
             chunk -= 1
@@ -292,7 +299,7 @@ def main():
         return
 
     peak, peak_src = measured_peak()
-    alg = algorithmic_bytes(w, L_R)
+    alg = algorithmic_bytes(w, L_R, variant)
     achieved = alg / (ms_step * 1e-3) / 1e9
     traffic = NCU_TRAFFIC_BYTES.get(w.name) if not args.layers else None
     line = {
@@ -301,6 +308,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
                    "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio, "keep_k": plan.k, "L_R": L_R,
+                   "variant": args.variant,
                    "storage": "bf16", "parallelism": f"dp{world} (independent caches per rank, no collective)",
                    "launch": info, "l2": "inputs (%.1f GB per rank) are far larger than the 126 MB L2; no flush"
                    % (2 * K.numel() * 2 / 1e9)},
@@ -312,7 +320,7 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
-    if not args.no_cpu and world == 1:
+    if not args.no_cpu and world == 1 and variant == 0:
         layers_bits = [(synth.to_bits(K[l * w.B:(l + 1) * w.B]), synth.to_bits(V[l * w.B:(l + 1) * w.B]))
                        for l in range(min(4, w.layers))]
         del K, V

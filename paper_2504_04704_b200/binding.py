@@ -291,6 +291,45 @@ def lagkv_gather(plan: Plan, K, V, idx, **kw):
     return plan.gather(K, V, idx, **kw)
 
 
+class ChunkedPrefill:
+    """Chunk-by-chunk compression during prefill (Section 4.2 of the paper: the first S + 2L
+    tokens, then L tokens per step, compressing between steps) on top of
+    ``lagkv_compress_append``.  The caller's model produces K/V rows chunk by chunk; ``feed``
+    appends them to the caches held here and runs the append pass, so the caches never grow
+    beyond ``capacity`` rows.  All sequences advance together."""
+
+    def __init__(self, B, H_kv, D, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1, capacity=None, device=0):
+        self.plan = Plan(B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof, device=device)
+        dev = self.plan._dev()
+        self.first = sink + 2 * lag                     # tokens of the first step
+        self.step = lag                                 # tokens of every later step
+        self.capacity = int(capacity if capacity is not None else sink + 4 * lag)
+        self.K = torch.zeros((B, H_kv, self.capacity, D), dtype=torch.bfloat16, device=dev)
+        self.V = torch.zeros_like(self.K)
+        self.seq_len = torch.zeros((B,), dtype=torch.int32, device=dev)
+        self.static_len = torch.full((B,), sink, dtype=torch.int32, device=dev)
+        self.ws = self.plan.new_workspace(2)
+        self.rows = 0                                   # stored rows (host copy of seq_len, all equal)
+        self.static = sink
+
+    def feed(self, K_new, V_new) -> None:
+        """Append ``[B, H, t, D]`` new rows (any t that fits) and compress."""
+        t = int(K_new.shape[2])
+        if self.rows + t > self.capacity:
+            raise ValueError("chunk does not fit the cache capacity")
+        self.K[:, :, self.rows:self.rows + t] = K_new
+        self.V[:, :, self.rows:self.rows + t] = V_new
+        self.seq_len += t
+        self.rows += t
+        self.plan.compress_append(self.K, self.V, self.seq_len, self.static_len, self.ws, max_new_chunks=2)
+        # the same integers on the host (Eq. 12): no device read-back needed between steps
+        new_rows = self.plan.compressed_len(self.rows, self.static)
+        rest = self.rows - self.static
+        if rest >= 2 * self.plan.cfg.lag:
+            self.static += (rest // self.plan.cfg.lag - 1) * self.plan.k
+        self.rows = new_rows
+
+
 class HostPrefill:
     """Prefill compression of a cache that lives in pinned HOST memory.
 

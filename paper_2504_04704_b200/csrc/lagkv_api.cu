@@ -192,7 +192,6 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
     if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
-    if (cfg->variant == LAGKV_VARIANT_L2NORM) return LAGKV_EUNSUPPORTED;
     if (cfg->D != 64 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
     if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
 
@@ -318,7 +317,7 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     P.n = int(rest / c.lag);
     P.rem = int(rest % c.lag);
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
-    P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : P.n;
+    P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : (c.variant == LAGKV_VARIANT_L2NORM ? P.n - 1 : P.n);
     P.total_slots = U * P.spu;
     P.stages = plan->pre.stages;
 
@@ -445,7 +444,8 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
     }
     long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
     const long long nparts = rest / c.lag;
-    const long long slots = U * (c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (nparts - 1) : nparts);
+    const long long slots = U * (c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (nparts - 1)
+                                 : c.variant == LAGKV_VARIANT_L2NORM ? nparts - 1 : nparts);
     info[0] = int(grid < slots ? grid : slots);
     info[1] = kKernels[plan->pre.kidx].NW * 32;
     info[2] = int(plan->pre.smem);

@@ -311,6 +311,36 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
     }
 }
 
+// L2-norm variant (Eq. 16): the Euclidean norm of every valid row of a staged K tile.
+template <class G, bool FULL>
+__device__ __forceinline__ void process_tile_l2(const uint4* __restrict__ tile, int nrows,
+                                                float* __restrict__ norm_out, int lane) {
+    const int cg = lane % G::LPR, rl = lane / G::LPR;
+    float p2[G::NV];
+#pragma unroll
+    for (int i = 0; i < G::NV; ++i) {
+        const int row = i * G::RPL + rl;
+        f32x2 s2 = 0ull;
+#pragma unroll
+        for (int v = 0; v < G::V; ++v) {
+            const uint4 q = tile[row * G::VPR + v * G::LPR + cg];
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const f32x2 z = bf2_to_f32x2(w[c]);
+                s2 = fma2(z, z, s2);
+            }
+        }
+        float lo, hi;
+        unpack2(s2, lo, hi);
+        p2[i] = lo + hi;
+    }
+    transposed_reduce<G::NV, G::LPR>(p2, cg);
+    constexpr int DUP = G::LPR / G::NV;
+    const int row = (cg / DUP) * G::RPL + rl;
+    if ((cg % DUP) == 0 && (FULL || row < nrows)) norm_out[row] = sqrtf(p2[0]);
+}
+
 // ------------------------------------------------------------------ coefficients of Eq. 9
 // Combine the per-warp min / max partials of one tensor (nw rows of [mn | mx], STAT words
 // each, packed bf16x2) and turn them into y = a * z + b for this lane's channels:
@@ -397,7 +427,7 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 
 // Selector for L <= NT * E: every thread keeps E consecutive tokens in registers; the key of
 // the k-th largest score is built bit by bit from block-wide counts.
-template <int NT, int E, class Sync, class Release>
+template <int NT, int E, bool SOFTMAX, class Sync, class Release>
 __device__ void select_in_registers(const float* sg0, const float* sg1, int L, int k,
                                     float* __restrict__ scores_g, int* kept, SelScratch& sc, int tid, Sync sync,
                                     Release release) {
@@ -433,35 +463,40 @@ __device__ void select_in_registers(const float* sg0, const float* sg1, int L, i
         m1 = fmaxf(m1, sc.red[1][w]);
     }
     // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
-    unsigned long long q0 = 0, q1 = 0;
+    float r0 = 0.f, r1 = 0.f;
+    if (SOFTMAX) {
+        unsigned long long q0 = 0, q1 = 0;
 #pragma unroll
-    for (int j = 0; j < E; ++j) {
-        x0[j] = softmax_exp(x0[j], m0);  // exp(-inf) = 0 for the padding
-        x1[j] = softmax_exp(x1[j], m1);
-        q0 += fx30(x0[j]);
-        q1 += fx30(x1[j]);
-    }
-    q0 = warp_sum_u64(q0);
-    q1 = warp_sum_u64(q1);
-    if (lane == 0) {
-        sc.redq[0][warp] = q0;
-        sc.redq[1][warp] = q1;
-    }
-    sync();
-    q0 = q1 = 0;
+        for (int j = 0; j < E; ++j) {
+            x0[j] = softmax_exp(x0[j], m0);  // exp(-inf) = 0 for the padding
+            x1[j] = softmax_exp(x1[j], m1);
+            q0 += fx30(x0[j]);
+            q1 += fx30(x1[j]);
+        }
+        q0 = warp_sum_u64(q0);
+        q1 = warp_sum_u64(q1);
+        if (lane == 0) {
+            sc.redq[0][warp] = q0;
+            sc.redq[1][warp] = q1;
+        }
+        sync();
+        q0 = q1 = 0;
 #pragma unroll
-    for (int w = 0; w < NWARP; ++w) {
-        q0 += sc.redq[0][w];
-        q1 += sc.redq[1][w];
+        for (int w = 0; w < NWARP; ++w) {
+            q0 += sc.redq[0][w];
+            q1 += sc.redq[1][w];
+        }
+        r0 = fx30_to_recip(q0);
+        r1 = fx30_to_recip(q1);
     }
-    const float r0 = fx30_to_recip(q0), r1 = fx30_to_recip(q1);
     // ---- Eq. 11, then the order-preserving integer image; padding gets the smallest key
     uint32_t key[E];
     uint32_t kor = 0u, kand = 0xffffffffu;
 #pragma unroll
     for (int j = 0; j < E; ++j) {
         const int t = t_lo + j;
-        const float sco = combine_scores(x0[j], r0, x1[j], r1);
+        // without the softmax (Eq. 16) sg0 holds the key norms and the score is minus the norm
+        const float sco = SOFTMAX ? combine_scores(x0[j], r0, x1[j], r1) : -x0[j];
         key[j] = t < L ? float_key(sco) : 0u;
         if (t < L) {
             kor |= key[j];
@@ -544,10 +579,18 @@ __device__ void select_in_registers(const float* sg0, const float* sg1, int L, i
 // Selector for any L: scores stay in shared memory (sg0 is overwritten with them), radix
 // select with 8 bits per pass.
 template <int NT, class Sync, class Release>
-__device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __restrict__ scores_g, int* kept,
-                                 SelScratch& sc, int tid, Sync sync, Release release) {
+__device__ void select_in_shared(float* sg0, float* sg1, int L, int k, bool softmax, float* __restrict__ scores_g,
+                                 int* kept, SelScratch& sc, int tid, Sync sync, Release release) {
     constexpr int NWARP = NT / 32;
     const int lane = tid & 31, warp = tid >> 5;
+    if (!softmax) {  // Eq. 16: sg0 holds the key norms, the score is minus the norm
+        for (int t = tid; t < L; t += NT) {
+            const float sco = -sg0[t];
+            sg0[t] = sco;
+            if (scores_g != nullptr) scores_g[t] = sco;
+        }
+        sync();
+    } else {
 
     // ---- softmax over the partition's tokens, K and V side by side (Eq. 10)
     float m0 = -INFINITY, m1 = -INFINITY;
@@ -601,6 +644,7 @@ __device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __
         if (scores_g != nullptr) scores_g[t] = sco;
     }
     sync();
+    }
 
     // ---- radix select: key of the k-th largest score, 8 bits per pass
     uint32_t prefix = 0, mask = 0;
@@ -691,14 +735,23 @@ __device__ void select_in_shared(float* sg0, float* sg1, int L, int k, float* __
 }
 
 // Dispatch: registers when the partition fits E tokens per thread, else shared memory.
+// softmax = false: the L2-norm variant (sg0 = key norms, sg1 unused).
 template <int NT, class Sync, class Release>
-__device__ __forceinline__ void score_and_select(float* sg0, float* sg1, int L, int k,
+__device__ __forceinline__ void score_and_select(float* sg0, float* sg1, int L, int k, bool softmax,
                                                  float* __restrict__ scores_g, int* kept, SelScratch& sc, int tid,
                                                  Sync sync, Release release) {
-    if (L <= NT * 6) select_in_registers<NT, 6>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
-    else if (L <= NT * 11) select_in_registers<NT, 11>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
-    else if (L <= NT * 22) select_in_registers<NT, 22>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
-    else select_in_shared<NT>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    if (!softmax) {
+        if (L <= NT * 22) select_in_registers<NT, 22, false>(sg0, sg0, L, k, scores_g, kept, sc, tid, sync, release);
+        else select_in_shared<NT>(sg0, sg1, L, k, false, scores_g, kept, sc, tid, sync, release);
+    } else if (L <= NT * 6) {
+        select_in_registers<NT, 6, true>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    } else if (L <= NT * 11) {
+        select_in_registers<NT, 11, true>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    } else if (L <= NT * 22) {
+        select_in_registers<NT, 22, true>(sg0, sg1, L, k, scores_g, kept, sc, tid, sync, release);
+    } else {
+        select_in_shared<NT>(sg0, sg1, L, k, true, scores_g, kept, sc, tid, sync, release);
+    }
 }
 
 // --------------------------------------------------------------------------- row copies
@@ -1006,7 +1059,7 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
                 scores_g = (P.mode == MODE_PREFILL)
                                ? P.scores_out + ((long long)u * n_c + p) * L
                                : P.scores_out + ((long long)u * P.max_chunks + p) * L;
-            score_and_select<G::NT>(sg0, sg1, L, k, scores_g, reinterpret_cast<int*>(sg1), sc, tid,
+            score_and_select<G::NT>(sg0, sg1, L, k, true, scores_g, reinterpret_cast<int*>(sg1), sc, tid,
                                      [] { __syncthreads(); }, [] {});
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {

@@ -76,11 +76,13 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     // Slot j of a unit.  LagKV (Eq. 7-9): partitions n-1 ... 0, each scored with the statistics
     // of the slot before it.  LocalKV (Eq. 14, Eq. 15): partitions n-2 ... 0, each visited
     // twice in a row, once for its own statistics and once to be scored with them.
+    // L2 norm (Eq. 16): partitions n-2 ... 0, each scored on its own from K alone.
     const int spu = P.spu;
-    const bool local_stats = P.variant == 1;
-    auto slot_part = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : n - 1 - j; };
-    auto slot_scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : j != 0; };  // needs the slot before it
-    const bool extra = s_first < s_hi && slot_scored(int(s_first % spu));
+    const bool local_stats = P.variant == 1, l2norm = P.variant == 2;
+    auto slot_part = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : (l2norm ? n - 2 - j : n - 1 - j); };
+    auto slot_scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : (l2norm || j != 0); };
+    auto slot_needs_prev = [&](int j) -> bool { return !l2norm && slot_scored(j); };
+    const bool extra = s_first < s_hi && slot_needs_prev(int(s_first % spu));
     const long long s_lo = extra ? s_first - 1 : s_first;
 
     const uint32_t full_bar = smem_u32(xbars), empty_bar = smem_u32(xbars + 2), copy_bar = smem_u32(xbars + 4);
@@ -120,7 +122,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
         bool dead = false;
 
-        const bool has_tiles = wj < ntiles;
+        const bool has_tiles = wj < ntiles && !(l2norm && tensor == 1);  // Eq. 16 reads K only
         // producer cursor: next tile to request, kept as (slots left, unit, partition, tile)
         // and advanced without divisions
         long long pleft = s_hi - s_lo;
@@ -186,7 +188,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             }
             float* sig = sgbase + (buf * 2 + tensor) * Lp;
 
-            for (int t = wj; t < ntiles; t += G::WT) {
+            for (int t = wj; has_tiles && t < ntiles; t += G::WT) {
                 if (dead) break;
                 if (!mbar_wait_bounded(bar_w + 8 * cslot, cparity)) {
                     dead = true;
@@ -197,7 +199,10 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                                                                    size_t(cslot) * G::TILE_BYTES);
                 const int nrows = min(G::TR, L - t * G::TR);
                 float* so = sig + t * G::TR;
-                if (nrows == G::TR) {
+                if (l2norm) {
+                    if (nrows == G::TR) process_tile_l2<G, true>(tile, nrows, so, lane);
+                    else process_tile_l2<G, false>(tile, nrows, so, lane);
+                } else if (nrows == G::TR) {
                     if (score) process_tile<G, true, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
                     else process_tile<G, false, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
                 } else {
@@ -239,7 +244,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             // ---- coefficients for the next (lower) partition from this one's statistics
             {
                 const int zero_range = make_coefficients<G>(stats_t, G::WT, cg, a2, b2);
-                if (zero_range != 0 && wj == 0 && rl == 0 && !dead && P.status != nullptr)
+                if (zero_range != 0 && wj == 0 && rl == 0 && !dead && !l2norm && P.status != nullptr)
                     atomicAdd(P.status + 2, zero_range);
             }
         }
@@ -269,7 +274,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 const uint32_t ebar = empty_bar + 8 * buf;
                 // the sigma buffer goes back to the streamers as soon as the selector has
                 // taken its values (called after a group barrier; one arrival is expected)
-                score_and_select<kWsSelThreads>(sg0, sg1, L, k, scores_g, kept, sc, etid, sync_sel, [&] {
+                score_and_select<kWsSelThreads>(sg0, sg1, L, k, !l2norm, scores_g, kept, sc, etid, sync_sel, [&] {
                     if (etid == 0) mbar_arrive(ebar);
                 });
                 // the kept rows themselves move in the gather phase at the end of the kernel;

@@ -262,10 +262,46 @@ def test_localkv_many_units_and_minimal(binding, oracle):
                 variant=binding.VARIANT_LOCALKV)
 
 
+L2_REL_TOL = 1e-5     # |gpu - oracle| <= L2_REL_TOL * |oracle| for the norm scores of Eq. 16
+
+
+@pytest.mark.parametrize("L,k,S_extra,B", [(64, 16, 60, 2), (100, 25, 7, 2), (256, 1, 255, 2), (1024, 256, 1008, 9),
+                                           (2048, 256, 100, 1), (37, 5, 36, 2)])
+def test_l2norm_prefill(binding, oracle, L, k, S_extra, B):
+    """L2-norm variant (Eq. 16): score = -||K row||, no softmax, V only gathered."""
+    H, D, sink = 3, 128, 4
+    n = 5 if L >= 512 else 9
+    S = sink + n * L + S_extra
+    K, V = synth.make_kv(B, H, S, D, seed=L + 9, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=binding.VARIANT_L2NORM, device=0)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill(K, V, ws, want_scores=True)
+    assert plan.read_status(ws)[0] == 0
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    ref = oracle.compress(Kb, Vb, sink, L, k, variant=oracle.VARIANT_L2NORM)
+    idx = out["idx"].cpu().numpy()
+    n_c = ref["n_c"]
+    assert out["L_R"] == ref["L_R"]
+    take = idx[..., None].astype(np.int64)
+    np.testing.assert_array_equal(synth.to_bits(out["K_out"]), np.take_along_axis(Kb, take, axis=2))
+    np.testing.assert_array_equal(synth.to_bits(out["V_out"]), np.take_along_axis(Vb, take, axis=2))
+    np.testing.assert_array_equal(idx[..., :sink], ref["idx"][..., :sink])
+    np.testing.assert_array_equal(idx[..., sink + n_c * k:], ref["idx"][..., sink + n_c * k:])
+    s32 = out["scores"].cpu().numpy()
+    err = np.abs(s32.astype(np.float64) - ref["scores"])
+    assert np.all(err <= L2_REL_TOL * np.abs(ref["scores"]))
+    own = np.sort(np.argsort(-s32, axis=-1, kind="stable")[..., :k], axis=-1) + (sink + np.arange(n_c) * L)[None, None, :, None]
+    got = idx[..., sink:sink + n_c * k].reshape(B, H, n_c, k)
+    np.testing.assert_array_equal(got, own)
+    want = ref["idx"][..., sink:sink + n_c * k].reshape(B, H, n_c, k)
+    for b, h, p in np.argwhere((got != want).any(-1)):
+        sc = ref["scores"][b, h, p]
+        kth = np.sort(sc)[::-1][k - 1]
+        diff = np.setxor1d(got[b, h, p], want[b, h, p]) - (sink + p * L)
+        assert np.all(np.abs(sc[diff] - kth) <= 2 * err[b, h, p].max())
+
+
 def test_variants_not_built_are_refused(binding):
-    with pytest.raises(binding.LagKVError) as e:
-        binding.Plan(1, 2, 128, 4, 64, variant=binding.VARIANT_L2NORM, device=0)
-    assert e.value.code == binding.LAGKV_EUNSUPPORTED
     plan = binding.Plan(1, 2, 128, 4, 64, keep_k=16, variant=binding.VARIANT_LOCALKV, device=0)
     K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
     seq = torch.tensor([300], dtype=torch.int32, device="cuda:0")
@@ -275,6 +311,9 @@ def test_variants_not_built_are_refused(binding):
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
     with pytest.raises(binding.LagKVError) as e:
         plan.tune(warps=2, tile_rows=16, stages=2, ctas_per_sm=1)     # the uniform kernel has no variants
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+    with pytest.raises(binding.LagKVError) as e:                      # nor partitions beyond its shared memory
+        binding.Plan(1, 2, 128, 4, 8192, keep_k=16, variant=binding.VARIANT_L2NORM, device=0)
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
 
 
@@ -392,6 +431,28 @@ def test_prefill_equals_incremental_on_gpu(binding, oracle):
     assert stat.tolist() == [sink + 4 * k] * B
     assert torch.equal(Kc[:, :, :one["L_R"]], one["K_out"])
     assert torch.equal(Vc[:, :, :one["L_R"]], one["V_out"])
+
+
+def test_chunked_prefill_driver_equals_one_shot(binding, oracle):
+    """Chunk-by-chunk prefill (first S + 2L tokens, then L per step) ends with the same cache as
+    one pass over the whole prompt, and with the oracle's."""
+    B, H, D, sink, L, k = 2, 3, 128, 16, 128, 32
+    total = sink + 2 * L + 5 * L + 77
+    K, V = synth.make_kv(B, H, total, D, seed=61, device="cuda:0")
+    drv = binding.ChunkedPrefill(B, H, D, sink, L, keep_k=k, device=0)
+    drv.feed(K[:, :, :drv.first], V[:, :, :drv.first])
+    pos = drv.first
+    while pos < total:
+        t = min(drv.step, total - pos)
+        drv.feed(K[:, :, pos:pos + t], V[:, :, pos:pos + t])
+        pos += t
+        assert drv.rows <= sink + 3 * L + 6 * k            # the cache stays short all along
+    assert drv.plan.read_status(drv.ws)[0] == 0
+    ref = oracle.compress(synth.to_bits(K), synth.to_bits(V), sink, L, k)
+    assert drv.rows == ref["L_R"] and drv.seq_len.tolist() == [ref["L_R"]] * B
+    assert drv.static_len.tolist() == [drv.static] * B
+    np.testing.assert_array_equal(synth.to_bits(drv.K[:, :, :drv.rows]), ref["K_out"])
+    np.testing.assert_array_equal(synth.to_bits(drv.V[:, :, :drv.rows]), ref["V_out"])
 
 
 # ----------------------------------------------------------------------- argument checks
