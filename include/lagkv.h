@@ -105,12 +105,14 @@ int64_t lagkv_compressed_len(lagkv_plan_t plan, int64_t seq_len, int64_t static_
 int32_t lagkv_keep_for_target(int64_t Ls, int32_t sink, int32_t lag, double target_C);
 
 /*
- * Bytes of workspace needed: the status block plus, for lagkv_compress_append(), room
- * for max_new_chunks*k kept indices per (b, h).  Pass 0 for prefill / gather only.
+ * Bytes of workspace needed: the status block plus, for lagkv_compress_append(), one counter
+ * per sequence (rounded up to 256 bytes) and room for max_new_chunks*k kept indices per
+ * (b, h).  Pass 0 for prefill / gather only.
  */
 size_t lagkv_workspace_bytes(lagkv_plan_t plan, int32_t max_new_chunks);
 
-/* Clear the status block (async memset on the stream).  Call once per workspace. */
+/* Clear the status block and the append counters (async memset on the stream).  Call once
+ * per workspace; the kernels leave the counters at zero. */
 int lagkv_workspace_init(lagkv_plan_t plan, void *workspace, size_t workspace_bytes,
                          void *cuda_stream);
 
@@ -169,12 +171,13 @@ int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64
  *   status_out  DEVICE int32[4] or NULL: receives the status block of this call (same
  *               meaning as lagkv_read_status(): [0] first device-side status, [1] detail,
  *               [2] zero-range channel count), written on cuda_stream after the kernels.
- * The call allocates nothing and frees nothing; it enqueues a 256-byte memset, the append
- * kernels and, if asked, a 16-byte device-to-device copy.
+ * The call allocates nothing and frees nothing; it enqueues a small memset (status block and
+ * counters), the append kernel and, if asked, a 16-byte device-to-device copy.
  *
- * Limit: 256 + B*H_kv*max_new_chunks*k*4 bytes must not exceed LAGKV_NOALLOC_SCRATCH_BYTES
- * when idx_out is NULL (the kept positions are parked in the scratch); with idx_out given
- * only the 256-byte status block is used.  Beyond the limit the call returns
+ * Limit: 256 + 256*ceil(B/64) + B*H_kv*max_new_chunks*k*4 bytes must not exceed
+ * LAGKV_NOALLOC_SCRATCH_BYTES when idx_out is NULL (the kept positions are parked in the
+ * scratch); with idx_out given only the first two terms (status block, one counter per
+ * sequence) are used.  Beyond the limit the call returns
  * LAGKV_ENOALLOC_LIMIT and touches nothing.
  *
  * First call on a device: the library looks up the device address of its array (once per

@@ -241,9 +241,13 @@ int32_t lagkv_keep_for_target(int64_t Ls, int32_t sink, int32_t lag, double targ
     return lag;
 }
 
+// Workspace layout: [status block | per-sequence head counters (append) | kept positions (append)]
+static size_t counter_words(const lagkv_plan_s* plan) { return (size_t(plan->cfg.B) + 63) / 64 * 64; }
+
 size_t lagkv_workspace_bytes(lagkv_plan_t plan, int32_t max_new_chunks) {
     if (plan == nullptr || max_new_chunks < 0) return 0;
     size_t bytes = kStatusWords * sizeof(int32_t);
+    if (max_new_chunks > 0) bytes += counter_words(plan) * sizeof(int32_t);
     bytes += size_t(plan->cfg.B) * plan->cfg.H_kv * size_t(max_new_chunks) * plan->k * sizeof(int32_t);
     return (bytes + 255) & ~size_t(255);
 }
@@ -253,8 +257,9 @@ int lagkv_workspace_init(lagkv_plan_t plan, void* workspace, size_t workspace_by
     if (workspace == nullptr || workspace_bytes < kStatusWords * sizeof(int32_t)) return LAGKV_EWORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
     DeviceGuard guard(plan->cfg.device);
-    if (cudaMemsetAsync(workspace, 0, kStatusWords * sizeof(int32_t), static_cast<cudaStream_t>(cuda_stream)) !=
-        cudaSuccess)
+    size_t clear = (kStatusWords + counter_words(plan)) * sizeof(int32_t);  // status block and head counters
+    if (clear > workspace_bytes) clear = kStatusWords * sizeof(int32_t);    // a prefill-only workspace
+    if (cudaMemsetAsync(workspace, 0, clear, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return LAGKV_ECUDA;
     return LAGKV_OK;
 }
@@ -345,7 +350,8 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
         return LAGKV_EINVAL;
     if (workspace == nullptr) return LAGKV_EWORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
-    const size_t need = idx_out ? kStatusWords * sizeof(int32_t) : lagkv_workspace_bytes(plan, max_new_chunks);
+    const size_t head = (kStatusWords + counter_words(plan)) * sizeof(int32_t);
+    const size_t need = idx_out ? head : lagkv_workspace_bytes(plan, max_new_chunks);
     if (workspace_bytes < need) return LAGKV_EWORKSPACE;
     const lagkv_config& c = plan->cfg;
     Strides st;
@@ -363,7 +369,8 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     P.seq_len = seq_len;
     P.static_len = static_len;
     P.status = static_cast<int32_t*>(workspace);
-    P.kept_pos = idx_out ? idx_out : static_cast<int32_t*>(workspace) + kStatusWords;
+    P.seq_done = static_cast<int32_t*>(workspace) + kStatusWords;
+    P.kept_pos = idx_out ? idx_out : P.seq_done + counter_words(plan);
     P.sb = st.sb;
     P.sh = st.sh;
     P.ss = st.ss;
@@ -385,8 +392,6 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)U), dim3(ke.NW * 32), args,
                          plan->app.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
-    lagkv_update_lengths_kernel<<<(c.B + 127) / 128, 128, 0, stream>>>(seq_len, static_len, c.B, c.lag, plan->k,
-                                                                       max_new_chunks, int(S_cap));
     return check_launch();
 }
 
@@ -519,14 +524,16 @@ extern "C" int lagkv_compress_append_noalloc(lagkv_plan_t plan, void* K_cache, v
     if (plan == nullptr || plan->cfg.device < 0 || max_new_chunks < 1) return LAGKV_EINVAL;
     if (reinterpret_cast<uintptr_t>(status_out) & 3u) return LAGKV_EINVAL;
     // without idx_out the kernel parks the kept positions in the scratch: that list must fit
-    const size_t need = idx_out ? kStatusWords * sizeof(int32_t) : lagkv_workspace_bytes(plan, max_new_chunks);
+    const size_t head = (kStatusWords + counter_words(plan)) * sizeof(int32_t);
+    const size_t need = idx_out ? head : lagkv_workspace_bytes(plan, max_new_chunks);
     if (need == 0 || need > size_t(LAGKV_NOALLOC_SCRATCH_BYTES)) return LAGKV_ENOALLOC_LIMIT;
     DeviceGuard guard(plan->cfg.device);
     void* scratch = noalloc_scratch_for(plan->cfg.device);
     if (scratch == nullptr) return LAGKV_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    // the array keeps what the previous call left: the status block has to start at zero
-    if (cudaMemsetAsync(scratch, 0, kStatusWords * sizeof(int32_t), stream) != cudaSuccess) return LAGKV_ECUDA;
+    // the array keeps what the previous call left: the status block and the per-sequence head
+    // counters have to start at zero
+    if (cudaMemsetAsync(scratch, 0, head, stream) != cudaSuccess) return LAGKV_ECUDA;
     const int rc = lagkv_compress_append(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out,
                                          scores_out, scratch, size_t(LAGKV_NOALLOC_SCRATCH_BYTES), stream);
     if (rc != LAGKV_OK) return rc;

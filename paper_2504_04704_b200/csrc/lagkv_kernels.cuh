@@ -41,6 +41,7 @@ struct Params {
     const int32_t* seq_len;     // append: device [B]
     const int32_t* static_len;  // append: device [B]
     int32_t* kept_pos;          // append: [U, max_chunks * k] pre-call positions of kept rows
+    int32_t* seq_done;          // append: [B] heads of a sequence that have finished (workspace, zero between calls)
     int32_t* status;            // status block
     long long sb, sh, ss;       // cache strides in elements
     long long total_slots;      // prefill: U * n
@@ -1111,6 +1112,18 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
             move_rows_inplace<G::NT, G::VPR>(ck, cv, P.ss, stat_rows + n_c * k, L + rem,
                                              [&](int j) { return src0 + j; }, tid);
         }
+        // The lengths of a sequence change once all of its heads are done: every head's CTA has
+        // read the old values by then.  The last one to finish writes the new ones and clears
+        // the counter for the next call.
+        if (tid == 0) {
+            const int b = u / P.H;
+            if (atomicAdd(P.seq_done + b, 1) == P.H - 1) {
+                P.seq_done[b] = 0;
+                const int ns = stat_rows + n_c * k;
+                const_cast<int32_t*>(P.static_len)[b] = ns;
+                const_cast<int32_t*>(P.seq_len)[b] = ns + L + rem;
+            }
+        }
     }
 
     // a wait that ran out may have left copies in flight: give them one more bounded chance
@@ -1118,22 +1131,6 @@ __global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
         const unsigned long long t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
     }
-}
-
-// append: lengths after the pass (run as a second launch so that every CTA of the main
-// kernel has read the old values)
-__global__ void lagkv_update_lengths_kernel(int32_t* seq_len, int32_t* static_len, int B, int L, int k,
-                                            int max_chunks, int S_cap) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    const int seq = seq_len[b], st = static_len[b];
-    const int rest = seq - st;
-    if (rest < 2 * L || st < 0 || seq > S_cap) return;
-    const int n = rest / L, rem = rest % L;
-    if (n - 1 > max_chunks) return;
-    const int ns = st + (n - 1) * k;
-    static_len[b] = ns;
-    seq_len[b] = ns + L + rem;
 }
 
 // identity pass (S_in < S + 2L) and plain strided -> contiguous copy
