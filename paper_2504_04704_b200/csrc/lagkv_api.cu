@@ -23,15 +23,19 @@ typedef size_t (*smem_fn_t)(int, int);
 // warps + 4 epilogue warps); the others are the uniform kernel that also serves appends.
 struct KernelEntry {
     int D, NW, TR;
+    int variant;  // enum lagkv_variant the kernel was compiled for (the uniform kernel: LagKV only)
     bool ws;
     stream_kernel_t fn;
     smem_fn_t smem;
 };
 
 #define LAGKV_ENTRY(D, V, NW, TR) \
-    { D, NW, TR, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+    { D, NW, TR, 0, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+#define LAGKV_WS_ENTRY1(D, V, NWS, TR, VAR) \
+    { D, NWS + kWsEpiWarps, TR, VAR, true, &lagkv_ws_kernel<Geo<D, V, NWS, TR>, VAR>, \
+      &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
 #define LAGKV_WS_ENTRY(D, V, NWS, TR) \
-    { D, NWS + kWsEpiWarps, TR, true, &lagkv_ws_kernel<Geo<D, V, NWS, TR>>, &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
+    LAGKV_WS_ENTRY1(D, V, NWS, TR, 0), LAGKV_WS_ENTRY1(D, V, NWS, TR, 1), LAGKV_WS_ENTRY1(D, V, NWS, TR, 2)
 
 const KernelEntry kKernels[] = {
     LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
@@ -45,9 +49,10 @@ const KernelEntry kKernels[] = {
 };
 constexpr int kNumKernels = int(sizeof(kKernels) / sizeof(kKernels[0]));
 
-int find_kernel(int D, int NW, int TR) {
+int find_kernel(int D, int NW, int TR, int variant) {
     for (int i = 0; i < kNumKernels; ++i)
-        if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR) return i;
+        if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR && kKernels[i].variant == variant)
+            return i;
     return -1;
 }
 
@@ -96,7 +101,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // Try one launch shape (NW = warps per CTA, 12 = the warp-specialised kernel).
 int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Shape* out) {
-    const int kidx = find_kernel(pl->cfg.D, NW, TR);
+    // the uniform kernel exists for LagKV only: a variant plan still gets it as its (refused) append shape
+    const int kidx = find_kernel(pl->cfg.D, NW, TR, NW == 8 + kWsEpiWarps ? pl->cfg.variant : 0);
     if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
     if (kKernels[kidx].ws && ctas != 1) return LAGKV_EUNSUPPORTED;
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
@@ -141,7 +147,7 @@ int choose_shape(lagkv_plan_s* pl) {
         uni[nu++] = {4, 32, 3, 2};
         uni[nu++] = {4, 32, 2, 2};
     }
-    uni[nu++] = {2, 16, 4, 6};
+    uni[nu++] = {2, 16, 3, 6};
     uni[nu++] = {2, 16, 3, 4};
     uni[nu++] = {2, 16, 2, 2};
     uni[nu++] = {2, 16, 2, 1};
@@ -149,7 +155,7 @@ int choose_shape(lagkv_plan_s* pl) {
     if (rc != LAGKV_OK) return rc;
     pl->pre = pl->app;
     const bool needs_ws = pl->cfg.variant != LAGKV_VARIANT_LAGKV;  // only that kernel knows the variants
-    if (L >= 128 || needs_ws) {
+    if (L >= 256 || needs_ws) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
         Shape sh;
         rc = first_fit(pl, ws, 3, &sh);

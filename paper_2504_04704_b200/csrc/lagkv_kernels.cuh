@@ -873,7 +873,8 @@ __device__ void move_rows_inplace(uint16_t* K, uint16_t* V, long long ss, int ds
 
 // ------------------------------------------------------------------------------- kernel
 template <class G>
-__global__ void __launch_bounds__(G::NT) lagkv_stream_kernel(const Params P) {
+// two-warp CTAs are meant to run six to an SM (short partitions): cap their registers for that
+__global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kernel(const Params P) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const int NS = P.stages;

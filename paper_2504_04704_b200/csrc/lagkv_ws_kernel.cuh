@@ -47,7 +47,9 @@ __host__ __device__ inline size_t ws_smem_total_bytes(int stages, int L) {
     return s + 128;                                         // alignment slack
 }
 
-template <class G>
+// VAR: 0 = LagKV, 1 = LocalKV, 2 = L2 norm (enum lagkv_variant), compiled apart so that the
+// LagKV kernel carries none of the other variants' code.
+template <class G, int VAR>
 __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(const Params P) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -78,7 +80,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     // twice in a row, once for its own statistics and once to be scored with them.
     // L2 norm (Eq. 16): partitions n-2 ... 0, each scored on its own from K alone.
     const int spu = P.spu;
-    const bool local_stats = P.variant == 1, l2norm = P.variant == 2;
+    constexpr bool local_stats = VAR == 1, l2norm = VAR == 2;
     auto slot_part = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : (l2norm ? n - 2 - j : n - 1 - j); };
     auto slot_scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : (l2norm || j != 0); };
     auto slot_needs_prev = [&](int j) -> bool { return !l2norm && slot_scored(j); };
