@@ -233,6 +233,14 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]);
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages,
                     int32_t ctas_per_sm);
 
+/*
+ * Self-test of the failure path: launches one warp that waits, with the same bounded wait the
+ * compress kernels use, on a barrier nothing will ever complete.  After about limit_ms
+ * (1..2000) the wait gives up and LAGKV_ETIMEOUT is recorded in the status block of
+ * `workspace` (read it with lagkv_read_status()); the device stays usable.  Asynchronous.
+ */
+int lagkv_selftest_bounded_wait(lagkv_plan_t plan, void *workspace, int32_t limit_ms, void *cuda_stream);
+
 const char *lagkv_status_string(int status);
 const char *lagkv_version(void);
 

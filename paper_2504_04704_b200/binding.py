@@ -29,7 +29,7 @@ EXPORTS = (
     "lagkv_keep_for_target", "lagkv_workspace_bytes", "lagkv_workspace_init",
     "lagkv_compress_prefill", "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
     "lagkv_read_status",
-    "lagkv_launch_info", "lagkv_plan_tune", "lagkv_status_string", "lagkv_version",
+    "lagkv_launch_info", "lagkv_plan_tune", "lagkv_selftest_bounded_wait", "lagkv_status_string", "lagkv_version",
 )
 
 
@@ -92,6 +92,8 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_launch_info.argtypes = [vp, i64, ctypes.POINTER(i32 * 4)]
     lib.lagkv_plan_tune.restype = ctypes.c_int
     lib.lagkv_plan_tune.argtypes = [vp, i32, i32, i32, i32]
+    lib.lagkv_selftest_bounded_wait.restype = ctypes.c_int
+    lib.lagkv_selftest_bounded_wait.argtypes = [vp, vp, i32, vp]
     lib.lagkv_status_string.restype = ctypes.c_char_p
     lib.lagkv_status_string.argtypes = [ctypes.c_int]
     lib.lagkv_version.restype = ctypes.c_char_p
@@ -184,6 +186,11 @@ class Plan:
         if rc == LAGKV_ECUDA or rc == LAGKV_EINVAL and st[0] != LAGKV_EINVAL:
             raise LagKVError(rc, "lagkv_read_status")
         return [int(v) for v in st]
+
+    def selftest_bounded_wait(self, workspace: torch.Tensor, limit_ms: int = 50) -> None:
+        """``lagkv_selftest_bounded_wait``: a wait that cannot succeed must end with LAGKV_ETIMEOUT."""
+        _check(self.lib.lagkv_selftest_bounded_wait(self.handle, _ptr(workspace), int(limit_ms),
+                                                    _stream(self._dev())), "lagkv_selftest_bounded_wait")
 
     def _check_cache(self, t: torch.Tensor, name: str):
         if t.dtype != torch.bfloat16 or not t.is_cuda or t.device.index != self.device:

@@ -479,6 +479,16 @@ int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t
     return LAGKV_OK;
 }
 
+int lagkv_selftest_bounded_wait(lagkv_plan_t plan, void* workspace, int32_t limit_ms, void* cuda_stream) {
+    if (plan == nullptr || workspace == nullptr || plan->cfg.device < 0 || limit_ms < 1 || limit_ms > 2000)
+        return LAGKV_EINVAL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
+    DeviceGuard guard(plan->cfg.device);
+    lagkv_selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<int32_t*>(workspace), 1000000ull * (unsigned long long)limit_ms);
+    return check_launch();
+}
+
 const char* lagkv_status_string(int status) {
     switch (status) {
         case LAGKV_OK: return "ok";

@@ -125,13 +125,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // Warp-collective bounded wait on an mbarrier phase: every lane polls, the warp leaves
 // together, and lane 0's clock decides when to give up (about one second).  Returns false
 // when the wait ran out.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  unsigned long long limit_ns = 1000000000ull) {
     if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
     const unsigned long long t0 = global_timer_ns();
     for (int it = 0; it < (1 << 24); ++it) {
         if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
         if ((it & 255) == 255) {
-            const int late = global_timer_ns() - t0 > 1000000000ull;
+            const int late = global_timer_ns() - t0 > limit_ns;
             if (__shfl_sync(0xffffffffu, late, 0)) break;
         }
     }
@@ -1132,6 +1133,17 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         const unsigned long long t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000000ull) { /* bounded drain delay */ }
     }
+}
+
+// Self-test of the bounded wait: one warp waits on an mbarrier phase that nothing will ever
+// complete; the wait must give up after limit_ns and the status block must say so.
+__global__ void lagkv_selftest_wait_kernel(int32_t* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) mbar_init(b, 1);
+    fence_mbar_init();
+    __syncthreads();
+    if (!mbar_wait_bounded(b, 0u, limit_ns) && threadIdx.x == 0) record_status(status, ST_ETIMEOUT, -1);
 }
 
 // identity pass (S_in < S + 2L) and plain strided -> contiguous copy

@@ -455,6 +455,24 @@ def test_chunked_prefill_driver_equals_one_shot(binding, oracle):
     np.testing.assert_array_equal(synth.to_bits(drv.V[:, :, :drv.rows]), ref["V_out"])
 
 
+def test_bounded_wait_gives_up_and_reports(binding):
+    """Failure path without a fault: a wait on a barrier that nothing completes runs out after
+    its limit, the status block says LAGKV_ETIMEOUT, and the same context goes on working."""
+    import time
+    plan = binding.Plan(1, 2, 128, 4, 64, keep_k=16, device=0)
+    ws = plan.new_workspace()
+    t0 = time.perf_counter()
+    plan.selftest_bounded_wait(ws, limit_ms=50)
+    st = plan.read_status(ws)
+    dt = time.perf_counter() - t0
+    assert st[0] == binding.LAGKV_ETIMEOUT and st[1] == -1
+    assert 0.04 < dt < 1.0
+    assert plan.read_status(ws)[0] == 0                      # reading cleared it
+    K, V = synth.make_kv(1, 2, 4 + 3 * 64, 128, seed=2, device="cuda:0")
+    out = plan.compress_prefill(K, V, ws)                    # the context is still usable
+    assert plan.read_status(ws)[0] == 0 and out["L_R"] == 4 + 2 * 16 + 64
+
+
 # ----------------------------------------------------------------------- argument checks
 def test_argument_errors(binding):
     with pytest.raises(binding.LagKVError) as e:
