@@ -455,6 +455,31 @@ def test_chunked_prefill_driver_equals_one_shot(binding, oracle):
     np.testing.assert_array_equal(synth.to_bits(drv.V[:, :, :drv.rows]), ref["V_out"])
 
 
+def test_host_prefill_pipeline_matches_direct_call(binding, oracle):
+    """The host end-to-end path (pinned host cache -> device chunks -> compress -> compacted rows
+    and indices back on the host, three streams, two staging slots) returns what one direct
+    call on the whole cache returns, and what the oracle says."""
+    B, H, D, sink, L, k = 6, 2, 128, 16, 256, 64
+    S = sink + 5 * L + 70
+    K, V = synth.make_kv(B, H, S, D, seed=71, device="cuda:0")
+    hp = binding.HostPrefill(B, H, D, S, sink, L, keep_k=k, chunk_B=2, device=0)
+    Kh, Vh = K.cpu().pin_memory(), V.cpu().pin_memory()
+    Ko = torch.zeros((B, H, hp.L_R, D), dtype=torch.bfloat16).pin_memory()
+    Vo = torch.zeros_like(Ko).pin_memory()
+    Io = torch.zeros((B, H, hp.L_R), dtype=torch.int32).pin_memory()
+    for _ in range(2):                                       # the second run reuses both slots
+        hp.run(Kh, Vh, Ko, Vo, Io)
+    torch.cuda.synchronize()
+    assert hp.h2d_bytes == 2 * K.numel() * 2 and hp.d2h_bytes == 2 * Ko.numel() * 2 + Io.numel() * 4
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    direct = plan.compress_prefill(K, V, plan.new_workspace())
+    assert torch.equal(Io, direct["idx"].cpu()) and torch.equal(Ko, direct["K_out"].cpu())
+    assert torch.equal(Vo, direct["V_out"].cpu())
+    ref = oracle.compress(synth.to_bits(K), synth.to_bits(V), sink, L, k)
+    np.testing.assert_array_equal(Io.numpy(), ref["idx"])
+    np.testing.assert_array_equal(synth.to_bits(Ko), ref["K_out"])
+
+
 def test_bounded_wait_gives_up_and_reports(binding):
     """Failure path without a fault: a wait on a barrier that nothing completes runs out after
     its limit, the status block says LAGKV_ETIMEOUT, and the same context goes on working."""
