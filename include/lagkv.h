@@ -55,10 +55,9 @@ enum lagkv_status {
 
 enum lagkv_variant {
     LAGKV_VARIANT_LAGKV = 0,   /* Eq. 7-11: statistics from the next partition        */
-    LAGKV_VARIANT_LOCALKV = 1, /* Eq. 14, Eq. 15: statistics from the partition itself;
-                                  lagkv_compress_prefill only (append: EUNSUPPORTED)   */
+    LAGKV_VARIANT_LOCALKV = 1, /* Eq. 14, Eq. 15: statistics from the partition itself */
     LAGKV_VARIANT_L2NORM = 2   /* Eq. 16: score = -||K row||_2, no softmax, V is only
-                                  gathered; lagkv_compress_prefill only                */
+                                  gathered                                             */
 };
 
 typedef struct {

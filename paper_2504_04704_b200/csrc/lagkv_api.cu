@@ -29,8 +29,12 @@ struct KernelEntry {
     smem_fn_t smem;
 };
 
-#define LAGKV_ENTRY(D, V, NW, TR) \
-    { D, NW, TR, 0, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+#define LAGKV_ENTRY1(D, V, NW, TR, VAR) \
+    { D, NW, TR, VAR, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>, VAR>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+#define LAGKV_ENTRY(D, V, NW, TR) LAGKV_ENTRY1(D, V, NW, TR, 0)
+/* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
+#define LAGKV_VARIANT_ENTRIES(D, V) \
+    LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
 #define LAGKV_WS_ENTRY1(D, V, NWS, TR, VAR) \
     { D, NWS + kWsEpiWarps, TR, VAR, true, &lagkv_ws_kernel<Geo<D, V, NWS, TR>, VAR>, \
       &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
@@ -44,6 +48,7 @@ const KernelEntry kKernels[] = {
     LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
     LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
     LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+    LAGKV_VARIANT_ENTRIES(128, 2), LAGKV_VARIANT_ENTRIES(64, 1), LAGKV_VARIANT_ENTRIES(256, 2),
     LAGKV_WS_ENTRY(128, 2, 8, 32), LAGKV_WS_ENTRY(128, 2, 8, 16), LAGKV_WS_ENTRY(64, 1, 8, 32),
     LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16),
 };
@@ -101,8 +106,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // Try one launch shape (NW = warps per CTA, 12 = the warp-specialised kernel).
 int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Shape* out) {
-    // the uniform kernel exists for LagKV only: a variant plan still gets it as its (refused) append shape
-    const int kidx = find_kernel(pl->cfg.D, NW, TR, NW == 8 + kWsEpiWarps ? pl->cfg.variant : 0);
+    const int kidx = find_kernel(pl->cfg.D, NW, TR, pl->cfg.variant);
     if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
     if (kKernels[kidx].ws && ctas != 1) return LAGKV_EUNSUPPORTED;
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
@@ -139,7 +143,7 @@ int choose_shape(lagkv_plan_s* pl) {
     const int L = pl->cfg.lag;
     Cand uni[8];
     int nu = 0;
-    if (L >= 1024) {
+    if (L >= 1024 && pl->cfg.variant == LAGKV_VARIANT_LAGKV) {  // eight-warp CTAs are compiled for LagKV only
         uni[nu++] = {8, 32, 3, 1};
         uni[nu++] = {8, 32, 2, 1};
     }
@@ -154,14 +158,12 @@ int choose_shape(lagkv_plan_s* pl) {
     int rc = first_fit(pl, uni, nu, &pl->app);
     if (rc != LAGKV_OK) return rc;
     pl->pre = pl->app;
-    const bool needs_ws = pl->cfg.variant != LAGKV_VARIANT_LAGKV;  // only that kernel knows the variants
-    if (L >= 256 || needs_ws) {
+    if (L >= 256) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
         Shape sh;
         rc = first_fit(pl, ws, 3, &sh);
         if (rc == LAGKV_ECUDA) return rc;
         if (rc == LAGKV_OK) pl->pre = sh;
-        else if (needs_ws) return LAGKV_EUNSUPPORTED;
     }
     return LAGKV_OK;
 }
@@ -349,7 +351,6 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
         plan->cfg.device < 0)
         return LAGKV_EINVAL;
     if (S_cap < 1 || S_cap > 0x7fffffffll - 65536 || max_new_chunks < 1) return LAGKV_EINVAL;
-    if (plan->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;  // variants: prefill only
     if (!aligned16(K_cache) || !aligned16(V_cache) || K_cache == V_cache) return LAGKV_EINVAL;
     if ((reinterpret_cast<uintptr_t>(idx_out) & 3u) || (reinterpret_cast<uintptr_t>(scores_out) & 3u) ||
         (reinterpret_cast<uintptr_t>(seq_len) & 3u) || (reinterpret_cast<uintptr_t>(static_len) & 3u))
@@ -473,7 +474,6 @@ int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t
                               stages ? stages : plan->pre.stages, ctas_per_sm ? ctas_per_sm : plan->pre.ctas_per_sm,
                               &sh);
     if (rc != LAGKV_OK) return rc;
-    if (!kKernels[sh.kidx].ws && plan->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
     plan->pre = sh;
     if (!kKernels[sh.kidx].ws) plan->app = sh;
     return LAGKV_OK;

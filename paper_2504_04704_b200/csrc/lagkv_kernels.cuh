@@ -873,8 +873,10 @@ __device__ void move_rows_inplace(uint16_t* K, uint16_t* V, long long ss, int ds
 }
 
 // ------------------------------------------------------------------------------- kernel
-template <class G>
-// two-warp CTAs are meant to run six to an SM (short partitions): cap their registers for that
+// VAR: 0 = LagKV, 1 = LocalKV, 2 = L2 norm (enum lagkv_variant), a template parameter so that the
+// LagKV kernel carries none of the other variants' code.
+// Two-warp CTAs are meant to run six to an SM (short partitions): their registers are capped for that.
+template <class G, int VAR>
 __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kernel(const Params P) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -895,11 +897,18 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     const int ntiles = (L + G::TR - 1) / G::TR;
     const bool contiguous = (P.ss == G::D);
 
+    // Slot j of a unit.  LagKV (Eq. 7-9): partitions n-1 ... 0, each scored with the statistics
+    // of the slot before it.  LocalKV (Eq. 14, Eq. 15): partitions n-2 ... 0, each visited twice
+    // in a row, once for its own statistics and once to be scored with them.  L2 norm (Eq. 16):
+    // partitions n-2 ... 0, each scored on its own from K alone.
+    constexpr bool local_stats = VAR == 1, l2norm = VAR == 2;
+
     // ---- which slots does this CTA walk?
     long long s_first, s_hi;  // owned slots [s_first, s_hi)
-    int n, stat_rows, unit_fixed = 0, rem = 0;
+    int n, spu, stat_rows, unit_fixed = 0, rem = 0;
     if (P.mode == MODE_PREFILL) {
         n = P.n;
+        spu = P.spu;
         stat_rows = P.sink;
         s_first = P.total_slots * blockIdx.x / gridDim.x;
         s_hi = P.total_slots * (blockIdx.x + 1) / gridDim.x;
@@ -920,16 +929,20 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
             if (tid == 0) record_status(P.status, ST_ECAPACITY, b);
             return;
         }
+        spu = local_stats ? 2 * (n - 1) : (l2norm ? n - 1 : n);
         s_first = 0;
-        s_hi = n;
+        s_hi = spu;
     }
     if (s_first >= s_hi) return;
-    // a range that starts in the middle of a unit first re-reads the partition above it
-    const bool extra = (P.mode == MODE_PREFILL) && (s_first % n) != 0;
+    auto part_of = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : (l2norm ? n - 2 - j : n - 1 - j); };
+    auto scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : (l2norm || j != 0); };
+    auto needs_prev = [&](int j) -> bool { return !l2norm && scored(j); };
+    // a range that starts at a slot that needs the one before it first re-reads that one
+    const bool extra = (P.mode == MODE_PREFILL) && needs_prev(int(s_first % spu));
     const long long s_lo = extra ? s_first - 1 : s_first;
 
-    auto slot_unit = [&](long long s) -> int { return P.mode == MODE_PREFILL ? int(s / n) : unit_fixed; };
-    auto slot_part = [&](long long s) -> int { return n - 1 - int(s % n); };
+    auto slot_unit = [&](long long s) -> int { return P.mode == MODE_PREFILL ? int(s / spu) : unit_fixed; };
+    auto slot_part = [&](long long s) -> int { return part_of(int(s % spu)); };
     const uint16_t* tbase = tensor ? P.V : P.K;
     auto unit_base = [&](const uint16_t* base, int u) -> const uint16_t* {
         return base + (long long)(u / P.H) * P.sb + (long long)(u % P.H) * P.sh;
@@ -945,7 +958,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     fence_proxy_async();
     __syncthreads();
 
-    const bool has_tiles = wj < ntiles;
+    const bool has_tiles = wj < ntiles && !(l2norm && tensor == 1);  // Eq. 16 reads K only
     long long ps = s_lo;  // producer cursor: next tile to request
     int pt = wj;
     int pslot = 0;
@@ -989,9 +1002,9 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     bool have_ref = false;
 
     for (long long s = s_lo; s < s_hi; ++s) {
-        const int u = slot_unit(s), p = slot_part(s);
-        const bool top = (p == n - 1);
-        const bool score = !top && s >= s_first && have_ref;
+        const int u = slot_unit(s), sj = int(s % spu), p = part_of(sj);
+        const bool first_of_unit = sj == 0, last_of_unit = sj == spu - 1;
+        const bool score = scored(sj) && s >= s_first && (have_ref || !needs_prev(sj));
 
         uint32_t mn[G::NWORD], mx[G::NWORD];
 #pragma unroll
@@ -1001,7 +1014,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         }
         float* sig = tensor ? sg1 : sg0;
 
-        for (int t = wj; t < ntiles; t += G::WT) {
+        for (int t = wj; has_tiles && t < ntiles; t += G::WT) {
             if (timed_out) break;  // nothing more is consumed once a wait has run out
             const uint32_t bar = bar_w + 8 * cslot;
             if (!mbar_wait_bounded(bar, cparity)) {
@@ -1016,7 +1029,10 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
                                                                size_t(cslot) * G::TILE_BYTES);
             const int nrows = min(G::TR, L - t * G::TR);
             float* so = sig + t * G::TR;
-            if (nrows == G::TR) {
+            if (l2norm) {
+                if (nrows == G::TR) process_tile_l2<G, true>(tile, nrows, so, lane);
+                else process_tile_l2<G, false>(tile, nrows, so, lane);
+            } else if (nrows == G::TR) {
                 if (score) process_tile<G, true, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
                 else process_tile<G, false, true>(tile, nrows, a2, b2, mn, mx, so, inv_D, inv_Dm, lane);
             } else {
@@ -1062,7 +1078,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
                 scores_g = (P.mode == MODE_PREFILL)
                                ? P.scores_out + ((long long)u * n_c + p) * L
                                : P.scores_out + ((long long)u * P.max_chunks + p) * L;
-            score_and_select<G::NT>(sg0, sg1, L, k, true, scores_g, reinterpret_cast<int*>(sg1), sc, tid,
+            score_and_select<G::NT>(sg0, sg1, L, k, !l2norm, scores_g, reinterpret_cast<int*>(sg1), sc, tid,
                                      [] { __syncthreads(); }, [] {});
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {
@@ -1080,23 +1096,24 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         // ---- coefficients for the next (lower) partition from this one's statistics
         {
             const int zero_range = make_coefficients<G>(stats + (tensor * G::WT) * 2 * (G::D / 2), G::WT, cg, a2, b2);
-            if (zero_range != 0 && wj == 0 && rl == 0 && P.status != nullptr) atomicAdd(P.status + 2, zero_range);
+            if (zero_range != 0 && wj == 0 && rl == 0 && !l2norm && P.status != nullptr)
+                atomicAdd(P.status + 2, zero_range);
             have_ref = true;
         }
 
-        // ---- rows copied verbatim (prefill): window with the top slot, sink with slot p = 0
+        // ---- rows copied verbatim (prefill): window with a unit's first slot, sink with its last
         if (P.mode == MODE_PREFILL && s >= s_first) {
             const uint16_t* uk = unit_base(P.K, u);
             const uint16_t* uv = unit_base(P.V, u);
             uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
             uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
             int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
-            if (top)
+            if (first_of_unit)
                 copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, stat_rows + (n - 1) * L, stat_rows + (n - 1) * k,
                                          L + P.rem, oi, tid);
-            if (p == 0) copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, 0, 0, stat_rows, oi, tid);
+            if (last_of_unit) copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, 0, 0, stat_rows, oi, tid);
         }
-        if (p == 0) have_ref = false;  // next slot belongs to another unit
+        if (last_of_unit) have_ref = false;  // next slot belongs to another unit
         __syncthreads();
     }
 

@@ -301,19 +301,14 @@ def test_l2norm_prefill(binding, oracle, L, k, S_extra, B):
         assert np.all(np.abs(sc[diff] - kth) <= 2 * err[b, h, p].max())
 
 
-def test_variants_not_built_are_refused(binding):
+def test_variant_shapes(binding):
+    """Variants run on the warp-specialised kernel and on the two uniform shapes compiled for
+    them; other shapes are refused, and a partition too long for any of them refuses the plan."""
     plan = binding.Plan(1, 2, 128, 4, 64, keep_k=16, variant=binding.VARIANT_LOCALKV, device=0)
-    K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
-    seq = torch.tensor([300], dtype=torch.int32, device="cuda:0")
-    stat = torch.tensor([4], dtype=torch.int32, device="cuda:0")
+    plan.tune(warps=2, tile_rows=16, stages=2, ctas_per_sm=1)
+    plan.tune(warps=12, tile_rows=32, stages=2, ctas_per_sm=1)
     with pytest.raises(binding.LagKVError) as e:
-        plan.compress_append(K, V, seq, stat, plan.new_workspace(4), max_new_chunks=4)
-    assert e.value.code == binding.LAGKV_EUNSUPPORTED
-    with pytest.raises(binding.LagKVError) as e:
-        plan.tune(warps=2, tile_rows=16, stages=2, ctas_per_sm=1)     # the uniform kernel has no variants
-    assert e.value.code == binding.LAGKV_EUNSUPPORTED
-    with pytest.raises(binding.LagKVError) as e:                      # nor partitions beyond its shared memory
-        binding.Plan(1, 2, 128, 4, 8192, keep_k=16, variant=binding.VARIANT_L2NORM, device=0)
+        plan.tune(warps=8, tile_rows=32, stages=2, ctas_per_sm=1)     # eight-warp CTAs: LagKV only
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
 
 
@@ -338,19 +333,20 @@ def test_gather(binding, oracle):
 
 
 # -------------------------------------------------------------------------------- append
-def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chunks, seed, tune=None, give_idx=True):
+def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chunks, seed, tune=None, give_idx=True,
+                variant=0):
     K, V = synth.make_kv(B, H, S_cap, D, seed=seed, device="cuda:0")
     Kb, Vb = synth.to_bits(K), synth.to_bits(V)
     seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
     stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
-    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0)
     if tune:
         plan.tune(**tune)
     ws = plan.new_workspace(max_chunks)
     idx_out = torch.full((B, H, max_chunks * k), -1, dtype=torch.int32, device="cuda:0") if give_idx else None
     plan.compress_append(K, V, seq_d, stat_d, ws, max_new_chunks=max_chunks, idx_out=idx_out)
     st = plan.read_status(ws)
-    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k)
+    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k, variant=variant)
     return dict(K=synth.to_bits(K), V=synth.to_bits(V), seq=seq_d.cpu().numpy(), stat=stat_d.cpu().numpy(),
                 idx=None if idx_out is None else idx_out.cpu().numpy(), status=st,
                 Kr=Kr, Vr=Vr, seq_r=seq_r, stat_r=stat_r, kept=kept, K0=Kb, V0=Vb)
@@ -392,6 +388,46 @@ def test_append_multi_chunk(binding, oracle, L, k, chunks):
     r = append_case(binding, oracle, 2, 2, 128, seq[1] + 9, sink, L, k, seq, stat, chunks, seed=L + k,
                     give_idx=(L != 96))
     check_append(r, 2)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("L,k,chunks", [(64, 16, 4), (256, 32, 3), (512, 128, 1)])
+def test_append_variants(binding, oracle, variant, L, k, chunks):
+    """LocalKV and L2-norm scoring in the incremental pass, ragged batch with a skipped sequence."""
+    sink = 8
+    stat = [sink, sink + 2 * k, sink]
+    seq = [stat[0] + (chunks + 1) * L + 3, stat[1] + (chunks + 1) * L + L - 1, stat[2] + 2 * L - 1]
+    r = append_case(binding, oracle, 3, 2, 128, seq[1] + 9, sink, L, k, seq, stat, chunks, seed=L + k + variant,
+                    variant=variant)
+    check_append(r, 3)
+    np.testing.assert_array_equal(r["K"][2], r["K0"][2])
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_prefill_equals_incremental_variants(binding, variant):
+    """Per variant: one-shot prefill (warp-specialised kernel) and block-wise appends (uniform
+    kernel) end with the same cache, bit for bit."""
+    B, H, D, sink, L, k = 2, 2, 128, 4, 256, 64
+    total = sink + 2 * L + 3 * L + 11
+    K, V = synth.make_kv(B, H, total, D, seed=52 + variant, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0)
+    assert plan.launch_info(total)["block"] == 384
+    ws = plan.new_workspace(1)
+    one = plan.compress_prefill(K, V, ws)
+    Kc = torch.zeros((B, H, total, D), dtype=torch.bfloat16, device="cuda:0")
+    Vc = torch.zeros_like(Kc)
+    seq = torch.zeros((B,), dtype=torch.int32, device="cuda:0")
+    stat = torch.full((B,), sink, dtype=torch.int32, device="cuda:0")
+    pos = 0
+    for step in [sink + 2 * L, 100, 156, 256, 200, 56 + 11]:
+        s = int(seq[0])
+        Kc[:, :, s:s + step], Vc[:, :, s:s + step] = K[:, :, pos:pos + step], V[:, :, pos:pos + step]
+        seq += step
+        pos += step
+        plan.compress_append(Kc, Vc, seq, stat, ws, max_new_chunks=1)
+    assert pos == total and plan.read_status(ws)[0] == 0
+    assert seq.tolist() == [one["L_R"]] * B
+    assert torch.equal(Kc[:, :, :one["L_R"]], one["K_out"]) and torch.equal(Vc[:, :, :one["L_R"]], one["V_out"])
 
 
 def test_append_capacity_error_leaves_sequence_alone(binding, oracle):
