@@ -1,7 +1,8 @@
 // LagKV prefill compress pass -- warp-specialised persistent kernel for sm_100a.
 //
-// Same slot walk as lagkv_stream_kernel (partitions of a unit in DESCENDING p, so the
-// statistics of partition p+1, Eq. 7 / Eq. 8, are at hand when p streams through), but the
+// Same slot walk as lagkv_stream_kernel (for LagKV: partitions of a unit in DESCENDING p, so
+// the statistics of partition p+1, Eq. 7 / Eq. 8, are at hand when p streams through; the
+// LocalKV and L2-norm variants of Section 4.3 have their own slot lists, see below), but the
 // CTA is split into three roles so that the streaming never stops:
 //
 //   * NW streaming warps (even: K, odd: V).  Each owns a ring of shared-memory tiles
@@ -11,7 +12,8 @@
 //     tensor meet once per partition on a named barrier to combine their min / max.
 //   * 3 select warps: softmax over the partition, K + V (Eq. 11) and top-k with ties to
 //     the lower index -- one partition behind the streamers, overlapped with them.  They
-//     record where the kept rows come from; the rows move in the gather phase below.
+//     publish where the kept rows come from; the rows are moved by the copy warp or, what it
+//     has not claimed by the end, in the gather phase.
 //   * 1 copy warp: moves rows global -> shared -> global with bulk async copies: the kept
 //     rows of partitions whose positions are published (bandwidth the streamers leave
 //     unused), and the rows that are kept verbatim (sink and sliding window) of ALL units,
@@ -30,7 +32,7 @@ namespace lagkv {
 
 constexpr int kWsEpiWarps = 4;      // 3 select warps + 1 copy warp
 constexpr int kWsSelThreads = 96;
-constexpr int kWsCopyRows = 32;     // rows per staged chunk of the verbatim copies
+constexpr int kWsCopyRows = 32;     // rows per staged chunk of the copy warp
 constexpr int kBarTensor = 1;       // named barriers 1, 2: streaming warps of K, of V
 constexpr int kBarSelect = 3;       // named barrier 3: the select warps
 
@@ -279,7 +281,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 score_and_select<kWsSelThreads>(sg0, sg1, L, k, !l2norm, scores_g, kept, sc, etid, sync_sel, [&] {
                     if (etid == 0) mbar_arrive(ebar);
                 });
-                // the kept rows themselves move in the gather phase at the end of the kernel;
+                // the kept rows themselves are moved by the copy warp or in the gather phase;
                 // here only their source positions are recorded: in idx_out when the caller
                 // wants it, else in the first word of each destination row of K_out
                 {
