@@ -223,12 +223,15 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]);
 /*
  * Tuning override of the launch shape: warps per CTA (2, 4 or 8 = the uniform kernel, used
  * for prefill and append alike; 12 = the warp-specialised prefill kernel with 8 streaming,
- * 3 select and 1 copy warp, which leaves the append shape alone), rows per staged tile
+ * 3 select and 1 copy warp; LAGKV_TUNE_PAIRS = the prefill kernel for partitions of at most
+ * 512 rows, four K/V warp pairs with an epilogue warp each, LagKV only; the last two leave
+ * the append shape alone), rows per staged tile
  * (16 or 32), ring stages per streaming warp (2..8) and resident CTAs per SM to size the
  * prefill grid for (>= 1; must be 1 with 12 warps).  A value of 0 keeps the current
  * choice.  Returns LAGKV_EUNSUPPORTED for a combination that was not compiled or does not
  * fit shared memory.
  */
+#define LAGKV_TUNE_PAIRS 100
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages,
                     int32_t ctas_per_sm);
 

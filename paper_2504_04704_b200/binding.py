@@ -21,6 +21,7 @@ LIB_PATH = Path(__file__).resolve().parent / "liblagkv_b200.so"
 LAGKV_OK, LAGKV_EINVAL, LAGKV_EUNSUPPORTED, LAGKV_EWORKSPACE, LAGKV_ECUDA, LAGKV_ETIMEOUT, LAGKV_ECAPACITY = range(7)
 LAGKV_ENOALLOC_LIMIT = 7
 NOALLOC_SCRATCH_BYTES = 1048576
+TUNE_PAIRS = 100          # lagkv_plan_tune(): the pair kernel for short partitions
 VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
 
 # every symbol include/lagkv.h declares

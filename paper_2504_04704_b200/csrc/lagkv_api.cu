@@ -11,6 +11,7 @@
 
 #include "lagkv_kernels.cuh"
 #include "lagkv_ws_kernel.cuh"
+#include "lagkv_pair_kernel.cuh"
 
 using namespace lagkv;
 
@@ -22,22 +23,28 @@ typedef size_t (*smem_fn_t)(int, int);
 // NW counts every warp of the CTA.  ws = warp-specialised prefill kernel (8 streaming
 // warps + 4 epilogue warps); the others are the uniform kernel that also serves appends.
 struct KernelEntry {
-    int D, NW, TR;
-    int variant;  // enum lagkv_variant the kernel was compiled for (the uniform kernel: LagKV only)
-    bool ws;
+    int D, NW, TR;  // NW: warps per CTA as named in lagkv_plan_tune() (LAGKV_TUNE_PAIRS for the pair kernel)
+    int variant;    // enum lagkv_variant the kernel was compiled for
+    bool ws;        // a persistent prefill-only kernel (warp-specialised or pair), one CTA per SM
+    int threads;    // CTA size
     stream_kernel_t fn;
     smem_fn_t smem;
 };
 
 #define LAGKV_ENTRY1(D, V, NW, TR, VAR) \
-    { D, NW, TR, VAR, false, &lagkv_stream_kernel<Geo<D, V, NW, TR>, VAR>, &smem_total_bytes<Geo<D, V, NW, TR>> }
+    { D, NW, TR, VAR, false, NW * 32, &lagkv_stream_kernel<Geo<D, V, NW, TR>, VAR>, \
+      &smem_total_bytes<Geo<D, V, NW, TR>> }
 #define LAGKV_ENTRY(D, V, NW, TR) LAGKV_ENTRY1(D, V, NW, TR, 0)
 /* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
 #define LAGKV_VARIANT_ENTRIES(D, V) \
     LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
 #define LAGKV_WS_ENTRY1(D, V, NWS, TR, VAR) \
-    { D, NWS + kWsEpiWarps, TR, VAR, true, &lagkv_ws_kernel<Geo<D, V, NWS, TR>, VAR>, \
+    { D, NWS + kWsEpiWarps, TR, VAR, true, (NWS + kWsEpiWarps) * 32, &lagkv_ws_kernel<Geo<D, V, NWS, TR>, VAR>, \
       &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
+/* the pair kernel for short partitions (LagKV) */
+#define LAGKV_PAIR_ENTRY(D, V, TR) \
+    { D, LAGKV_TUNE_PAIRS, TR, 0, true, (2 * kPairs + kPairs) * 32, &lagkv_pair_kernel<Geo<D, V, 2 * kPairs, TR>>, \
+      &pair_smem_total_bytes<Geo<D, V, 2 * kPairs, TR>> }
 #define LAGKV_WS_ENTRY(D, V, NWS, TR) \
     LAGKV_WS_ENTRY1(D, V, NWS, TR, 0), LAGKV_WS_ENTRY1(D, V, NWS, TR, 1), LAGKV_WS_ENTRY1(D, V, NWS, TR, 2)
 
@@ -48,6 +55,7 @@ const KernelEntry kKernels[] = {
     LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
     LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
     LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+    LAGKV_PAIR_ENTRY(128, 2, 32), LAGKV_PAIR_ENTRY(128, 2, 16), LAGKV_PAIR_ENTRY(64, 1, 32), LAGKV_PAIR_ENTRY(256, 2, 16),
     LAGKV_VARIANT_ENTRIES(128, 2), LAGKV_VARIANT_ENTRIES(64, 1), LAGKV_VARIANT_ENTRIES(256, 2),
     LAGKV_WS_ENTRY(128, 2, 8, 32), LAGKV_WS_ENTRY(128, 2, 8, 16), LAGKV_WS_ENTRY(64, 1, 8, 32),
     LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16),
@@ -109,6 +117,7 @@ int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Sha
     const int kidx = find_kernel(pl->cfg.D, NW, TR, pl->cfg.variant);
     if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
     if (kKernels[kidx].ws && ctas != 1) return LAGKV_EUNSUPPORTED;
+    if (NW == LAGKV_TUNE_PAIRS && pl->cfg.lag > 512) return LAGKV_EUNSUPPORTED;  // one warp selects: L <= 512
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
     if (smem > size_t(pl->max_smem_optin)) return LAGKV_EUNSUPPORTED;
     if ((smem + 1024) * size_t(ctas) > size_t(kSmemPerSm)) return LAGKV_EUNSUPPORTED;
@@ -338,7 +347,7 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
     if (grid > P.total_slots) grid = P.total_slots;
     void* args[] = {&P};
-    if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)grid), dim3(ke.NW * 32), args,
+    if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)grid), dim3(ke.threads), args,
                          plan->pre.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
     return check_launch();
@@ -459,7 +468,7 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
     const long long slots = U * (c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (nparts - 1)
                                  : c.variant == LAGKV_VARIANT_L2NORM ? nparts - 1 : nparts);
     info[0] = int(grid < slots ? grid : slots);
-    info[1] = kKernels[plan->pre.kidx].NW * 32;
+    info[1] = kKernels[plan->pre.kidx].threads;
     info[2] = int(plan->pre.smem);
     info[3] = 1;
     return LAGKV_OK;

@@ -246,6 +246,53 @@ def test_power_of_two_channel_rescale_is_bit_invariant(binding):
     assert torch.equal(a["scores"], b["scores"])
 
 
+# --------------------------------------------------------------------------- pair kernel
+PAIRS = dict(warps=100, tile_rows=32, stages=2, ctas_per_sm=1)
+
+
+@pytest.mark.parametrize("L,k,S_extra,B", [(64, 4, 60, 2), (64, 16, 0, 40), (100, 25, 7, 2), (72, 72, 0, 2), (128, 32, 100, 3),
+                                           (256, 1, 255, 2), (512, 128, 3, 2), (500, 250, 499, 5), (37, 5, 36, 2),
+                                           (2, 1, 1, 2)])
+def test_pair_kernel_prefill(binding, oracle, L, k, S_extra, B):
+    """The kernel for short partitions (four independent K/V warp pairs per CTA, selection by one
+    warp): tile counts from 1 to 16 per partition, ragged tiles, remainders, idle pairs."""
+    n = 5 if L >= 500 else 9
+    run_prefill(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 3, tune=PAIRS)
+
+
+@pytest.mark.parametrize("D,tile_rows", [(64, 32), (256, 16), (128, 16)])
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_pair_kernel_head_dims(binding, oracle, D, tile_rows, ddof):
+    run_prefill(binding, oracle, 2, 4, D, 16 + 6 * 128 + 37, 16, 128, 32, seed=D + ddof + 1, ddof=ddof,
+                tune=dict(PAIRS, tile_rows=tile_rows))
+
+
+@pytest.mark.parametrize("layout", ["bshd", "padded"])
+def test_pair_kernel_strided_and_many_units(binding, oracle, layout):
+    run_prefill(binding, oracle, 37, 5, 128, 3 + 6 * 64 + 5, 3, 64, 16, seed=79, layout=layout, tune=PAIRS)
+
+
+def test_pair_kernel_same_bits_as_other_kernels(binding):
+    """Scores and selection do not depend on which kernel ran: bit-identical outputs from the
+    pair kernel, the warp-specialised kernel and the uniform kernel."""
+    B, H, D, sink, L, k = 3, 4, 128, 8, 256, 64
+    S = sink + 7 * L + 99
+    K, V = synth.make_kv(B, H, S, D, seed=81, device="cuda:0")
+    outs = []
+    for tune in (PAIRS, dict(warps=12, tile_rows=32, stages=2, ctas_per_sm=1), dict(warps=4, tile_rows=32, stages=2, ctas_per_sm=2),
+                 dict(warps=2, tile_rows=16, stages=3, ctas_per_sm=4)):
+        plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+        plan.tune(**tune)
+        ws = plan.new_workspace()
+        outs.append(plan.compress_prefill(K, V, ws, want_scores=True))
+        assert plan.read_status(ws)[0] == 0
+    for o in outs[1:]:
+        assert torch.equal(o["scores"], outs[0]["scores"]) and torch.equal(o["idx"], outs[0]["idx"])
+        assert torch.equal(o["K_out"], outs[0]["K_out"]) and torch.equal(o["V_out"], outs[0]["V_out"])
+    with pytest.raises(binding.LagKVError):                  # one warp selects: L <= 512 only
+        binding.Plan(1, 2, 128, 4, 1024, keep_k=16, device=0).tune(**PAIRS)
+
+
 # ------------------------------------------------------------------------------ variants
 @pytest.mark.parametrize("L,k,S_extra,B", [(64, 16, 60, 2), (100, 25, 7, 2), (256, 1, 255, 2), (512, 128, 3, 2),
                                            (1024, 256, 1008, 9), (2048, 256, 100, 1), (37, 5, 36, 2), (2, 1, 1, 2)])
