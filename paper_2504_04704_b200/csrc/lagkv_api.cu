@@ -86,6 +86,8 @@ struct lagkv_plan_s {
     int sm_count;
     int max_smem_optin;
     Shape pre;        // kernel used by lagkv_compress_prefill
+    Shape pair;       // pair kernel, preferred for short partitions with enough of them (kidx < 0: none)
+    bool tuned;       // lagkv_plan_tune() fixed the prefill kernel: no switching by size
     Shape app;        // kernel used by lagkv_compress_append (always the uniform kernel)
 };
 
@@ -167,6 +169,8 @@ int choose_shape(lagkv_plan_s* pl) {
     int rc = first_fit(pl, uni, nu, &pl->app);
     if (rc != LAGKV_OK) return rc;
     pl->pre = pl->app;
+    pl->pair.kidx = -1;
+    pl->tuned = false;
     if (L >= 256) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
         Shape sh;
@@ -174,7 +178,23 @@ int choose_shape(lagkv_plan_s* pl) {
         if (rc == LAGKV_ECUDA) return rc;
         if (rc == LAGKV_OK) pl->pre = sh;
     }
+    // Short partitions, few rows kept: four independent streams per CTA beat one partition at a
+    // time (measured on the Ls = 65536 sweep).  Whether there are enough partitions to feed
+    // them is known only at the call.
+    if (pl->cfg.variant == LAGKV_VARIANT_LAGKV && ((L <= 128 && 4 * pl->k <= L) || (L <= 256 && 8 * pl->k <= L))) {
+        const Cand pr[] = {{LAGKV_TUNE_PAIRS, 32, 2, 1}, {LAGKV_TUNE_PAIRS, 16, 2, 1}};
+        Shape sh;
+        rc = first_fit(pl, pr, 2, &sh);
+        if (rc == LAGKV_ECUDA) return rc;
+        if (rc == LAGKV_OK) pl->pair = sh;
+    }
     return LAGKV_OK;
+}
+
+// The prefill kernel for a call with `slots` (unit, partition) slots.
+const Shape& prefill_shape(const lagkv_plan_s* pl, long long slots) {
+    if (!pl->tuned && pl->pair.kidx >= 0 && slots >= 6ll * kPairs * pl->sm_count) return pl->pair;
+    return pl->pre;
 }
 
 struct Strides {
@@ -341,14 +361,15 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
     P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : (c.variant == LAGKV_VARIANT_L2NORM ? P.n - 1 : P.n);
     P.total_slots = U * P.spu;
-    P.stages = plan->pre.stages;
+    const Shape& shape = prefill_shape(plan, P.total_slots);
+    P.stages = shape.stages;
 
-    const KernelEntry& ke = kKernels[plan->pre.kidx];
-    long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
+    const KernelEntry& ke = kKernels[shape.kidx];
+    long long grid = (long long)plan->sm_count * shape.ctas_per_sm;
     if (grid > P.total_slots) grid = P.total_slots;
     void* args[] = {&P};
     if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)grid), dim3(ke.threads), args,
-                         plan->pre.smem, stream) != cudaSuccess)
+                         shape.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
     return check_launch();
 }
@@ -463,13 +484,14 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
         info[3] = S_in > 0 ? 1 : 0;
         return LAGKV_OK;
     }
-    long long grid = (long long)plan->sm_count * plan->pre.ctas_per_sm;
     const long long nparts = rest / c.lag;
     const long long slots = U * (c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (nparts - 1)
                                  : c.variant == LAGKV_VARIANT_L2NORM ? nparts - 1 : nparts);
+    const Shape& shape = prefill_shape(plan, slots);
+    const long long grid = (long long)plan->sm_count * shape.ctas_per_sm;
     info[0] = int(grid < slots ? grid : slots);
-    info[1] = kKernels[plan->pre.kidx].threads;
-    info[2] = int(plan->pre.smem);
+    info[1] = kKernels[shape.kidx].threads;
+    info[2] = int(shape.smem);
     info[3] = 1;
     return LAGKV_OK;
 }
@@ -484,6 +506,7 @@ int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t
                               &sh);
     if (rc != LAGKV_OK) return rc;
     plan->pre = sh;
+    plan->tuned = true;
     if (!kKernels[sh.kidx].ws) plan->app = sh;
     return LAGKV_OK;
 }
