@@ -4,14 +4,13 @@
  * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
  * LagKV compression pass (arXiv 2504.04704, Section 2.2 "LagKV") computes.  It is
  * used by the tests, by the smoke check and by the benchmark's CPU-baseline leg to
- * judge the CUDA library; the CUDA library never calls it and shares no code with it.
+ * check the CUDA library; the CUDA library never calls it and shares no code with it.
  *
  * Every step is written in the order the paper's Methodology lists it, one loop per
  * step, with no blocking, fusion or reordering.  Inputs are bf16 bit patterns
  * (uint16_t); each is widened exactly to double before any arithmetic.
  *
- * Readings taken where the paper leaves a choice (the same list is kept in the
- * design document):
+ * Readings taken where the paper leaves a choice:
  *   - min/max are taken over the tokens of the reference partition, one pair per
  *     channel (Eq. 7, Eq. 8: "min_seq", "max_seq").
  *   - "Std." is the standard deviation over the head_dim channels of one token,

@@ -1,7 +1,7 @@
 """GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle
 on the same seeded bf16 inputs.
 
-Bars (see also the design document):
+Bars:
   * per-token scores within 1e-4 absolute of the oracle (binding) and, tighter, within
     SCORE_REL_TOL of the mean score 2/L;
   * kept index sets identical to the oracle's, except partitions where the oracle's own
