@@ -84,7 +84,7 @@ typedef struct {
 int lagkv_plan(const lagkv_config *cfg, lagkv_plan_t *out);
 void lagkv_plan_destroy(lagkv_plan_t plan);
 
-/* k, the rows kept per compressed partition ("only rL tokens will be kept"). */
+/* k, the rows kept per compressed partition (r*L, text before Eq. 12). */
 int32_t lagkv_keep_count(lagkv_plan_t plan);
 
 /*

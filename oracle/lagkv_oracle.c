@@ -12,7 +12,7 @@
  *
  * Readings taken where the paper leaves a choice:
  *   - min/max are taken over the tokens of the reference partition, one pair per
- *     channel (Eq. 7, Eq. 8: "min_seq", "max_seq").
+ *     channel (Eq. 7, Eq. 8 reduce over the sequence axis).
  *   - "Std." is the standard deviation over the head_dim channels of one token,
  *     two-pass, divisor (D - ddof); ddof is a parameter (1 = sample std, 0 =
  *     population std).  The paper does not say which: PARITY UNPINNED for ddof.
@@ -67,7 +67,7 @@ void lagkv_oracle_set_threads(int n)
 #endif
 }
 
-/* Retained tokens per partition: "only rL tokens will be kept" (text before Eq. 12). */
+/* Retained tokens per partition: r*L of the L tokens stay (text before Eq. 12). */
 int64_t lagkv_oracle_keep_count(double r, int64_t L)
 {
     int64_t k = (int64_t)ceil(r * (double)L - 1e-9);
@@ -81,7 +81,7 @@ int64_t lagkv_oracle_keep_count(double r, int64_t L)
  * (sink + already compressed part) are left alone.  With static_len = S this is
  * Eq. 12:  L_R = S + rL*(floor((Ls-S)/L) - 1) + L + Mod(Ls-S, L);
  * below 2L of remaining rows the pass is skipped (third bullet of Section 2.2,
- * and "for the case Ls < S+2L, the compression ratio is zero").
+ * and the remark after Eq. 13 that shorter sequences are not compressed at all).
  */
 int64_t lagkv_oracle_compressed_len(int64_t seq_len, int64_t static_len, int64_t L, int64_t k)
 {

@@ -99,7 +99,7 @@ def test_eq12_table(oracle, args, want):
 
 
 def test_skip_below_two_lags(oracle):
-    # "For the case Ls < S+2L, the compression ratio is zero."
+    # remark after Eq. 13: a sequence shorter than S + 2L is not compressed at all
     for Ls in (0, 5, 16 + 2 * 32 - 1):
         assert oracle.compressed_len(Ls, 16, 32, 8) == Ls
     assert oracle.compressed_len(16 + 2 * 32, 16, 32, 8) == 16 + 8 + 32
