@@ -119,14 +119,16 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
 
     if (warp < G::NW) {
         // =============================================================== streaming warps
-        const int tensor = warp & 1, wj = warp >> 1;
+        // even warps stream K, odd warps V; the L2-norm variant reads K only and puts every warp on it
+        constexpr int WTE = l2norm ? G::NW : G::WT;  // warps that share a tensor's tiles
+        const int tensor = l2norm ? 0 : (warp & 1), wj = l2norm ? warp : (warp >> 1);
         const int cg = lane % G::LPR, rl = lane / G::LPR;
         const uint16_t* tbase = tensor ? P.V : P.K;
         const uint32_t ring_w = smem_u32(ring) + uint32_t(warp) * NS * G::TILE_BYTES;
         const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
         bool dead = false;
 
-        const bool has_tiles = wj < ntiles && !(l2norm && tensor == 1);  // Eq. 16 reads K only
+        const bool has_tiles = wj < ntiles;
         // producer cursor: next tile to request, kept as (slots left, unit, partition, tile)
         // and advanced without divisions
         long long pleft = s_hi - s_lo;
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 for (int r = lane; r < rows; r += 32)
                     bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
             }
-            pt += G::WT;
+            pt += WTE;
             if (pt >= ntiles) {  // next slot of this unit, or the first slot of the next unit
                 pt = wj;
                 --pleft;
@@ -192,7 +194,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             }
             float* sig = sgbase + (buf * 2 + tensor) * Lp;
 
-            for (int t = wj; has_tiles && t < ntiles; t += G::WT) {
+            for (int t = wj; has_tiles && t < ntiles; t += WTE) {
                 if (dead) break;
                 if (!mbar_wait_bounded(bar_w + 8 * cslot, cparity)) {
                     dead = true;
@@ -241,7 +243,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                         st[STAT_WORDS + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
                     }
             }
-            named_bar_sync(kBarTensor + tensor, G::WT * 32);
+            named_bar_sync(kBarTensor + tensor, WTE * 32);
             // sigma of this tensor is complete: hand the slot to the select warps
             if (lane == 0) mbar_arrive(full_bar + 8 * buf);
 
