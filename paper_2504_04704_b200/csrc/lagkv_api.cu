@@ -9,58 +9,36 @@
 #include <mutex>
 #include <new>
 
-#include "lagkv_kernels.cuh"
-#include "lagkv_ws_kernel.cuh"
-#include "lagkv_pair_kernel.cuh"
+#include "lagkv_aux_kernels.cuh"
+#include "lagkv_tables.h"
 
 using namespace lagkv;
 
 namespace {
 
-typedef void (*stream_kernel_t)(const Params);
-typedef size_t (*smem_fn_t)(int, int);
-
-// NW counts every warp of the CTA.  ws = warp-specialised prefill kernel (8 streaming
-// warps + 4 epilogue warps); the others are the uniform kernel that also serves appends.
-struct KernelEntry {
-    int D, NW, TR;  // NW: warps per CTA as named in lagkv_plan_tune() (LAGKV_TUNE_PAIRS for the pair kernel)
-    int variant;    // enum lagkv_variant the kernel was compiled for
-    bool ws;        // a persistent prefill-only kernel (warp-specialised or pair), one CTA per SM
-    int threads;    // CTA size
-    stream_kernel_t fn;
-    smem_fn_t smem;
+// every compiled kernel: the three tables live in translation units of their own
+struct KernelTable {
+    const KernelEntry* e[160];
+    int n = 0;
+    KernelTable() {
+        const KernelEntry* t;
+        int c = uniform_kernels(&t);
+        for (int i = 0; i < c; ++i) e[n++] = t + i;
+        c = ws_kernels(&t);
+        for (int i = 0; i < c; ++i) e[n++] = t + i;
+        c = pair_kernels(&t);
+        for (int i = 0; i < c; ++i) e[n++] = t + i;
+    }
 };
-
-#define LAGKV_ENTRY1(D, V, NW, TR, VAR) \
-    { D, NW, TR, VAR, false, NW * 32, &lagkv_stream_kernel<Geo<D, V, NW, TR>, VAR>, \
-      &smem_total_bytes<Geo<D, V, NW, TR>> }
-#define LAGKV_ENTRY(D, V, NW, TR) LAGKV_ENTRY1(D, V, NW, TR, 0)
-/* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
-#define LAGKV_VARIANT_ENTRIES(D, V) \
-    LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
-#define LAGKV_WS_ENTRY1(D, V, NWS, TR, VAR) \
-    { D, NWS + kWsEpiWarps, TR, VAR, true, (NWS + kWsEpiWarps) * 32, &lagkv_ws_kernel<Geo<D, V, NWS, TR>, VAR>, \
-      &ws_smem_total_bytes<Geo<D, V, NWS, TR>> }
-/* the pair kernel for short partitions (LagKV) */
-#define LAGKV_PAIR_ENTRY(D, V, TR) \
-    { D, LAGKV_TUNE_PAIRS, TR, 0, true, (2 * kPairs + kPairs) * 32, &lagkv_pair_kernel<Geo<D, V, 2 * kPairs, TR>>, \
-      &pair_smem_total_bytes<Geo<D, V, 2 * kPairs, TR>> }
-#define LAGKV_WS_ENTRY(D, V, NWS, TR) \
-    LAGKV_WS_ENTRY1(D, V, NWS, TR, 0), LAGKV_WS_ENTRY1(D, V, NWS, TR, 1), LAGKV_WS_ENTRY1(D, V, NWS, TR, 2)
-
-const KernelEntry kKernels[] = {
-    LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
-    LAGKV_ENTRY(128, 2, 8, 16), LAGKV_ENTRY(128, 2, 4, 16), LAGKV_ENTRY(128, 2, 2, 16),
-    LAGKV_ENTRY(64, 1, 8, 32),  LAGKV_ENTRY(64, 1, 4, 32),  LAGKV_ENTRY(64, 1, 2, 32),
-    LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
-    LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
-    LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
-    LAGKV_PAIR_ENTRY(128, 2, 32), LAGKV_PAIR_ENTRY(128, 2, 16), LAGKV_PAIR_ENTRY(64, 1, 32), LAGKV_PAIR_ENTRY(256, 2, 16),
-    LAGKV_VARIANT_ENTRIES(128, 2), LAGKV_VARIANT_ENTRIES(64, 1), LAGKV_VARIANT_ENTRIES(256, 2),
-    LAGKV_WS_ENTRY(128, 2, 8, 32), LAGKV_WS_ENTRY(128, 2, 8, 16), LAGKV_WS_ENTRY(64, 1, 8, 32),
-    LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16),
+const KernelTable& table() {
+    static const KernelTable t;
+    return t;
+}
+struct KernelRef {  // kKernels[i] reads like an array
+    const KernelEntry& operator[](int i) const { return *table().e[i]; }
 };
-constexpr int kNumKernels = int(sizeof(kKernels) / sizeof(kKernels[0]));
+const KernelRef kKernels;
+#define kNumKernels (table().n)
 
 int find_kernel(int D, int NW, int TR, int variant) {
     for (int i = 0; i < kNumKernels; ++i)

@@ -1,0 +1,19 @@
+// Instantiations of the pair kernel for short partitions (LagKV).
+#include "lagkv_tables.h"
+
+namespace lagkv {
+namespace {
+#define LAGKV_PAIR_ENTRY(D, V, TR) \
+    { D, LAGKV_TUNE_PAIRS, TR, 0, true, (2 * kPairs + kPairs) * 32, &lagkv_pair_kernel<Geo<D, V, 2 * kPairs, TR>>, \
+      &pair_smem_total_bytes<Geo<D, V, 2 * kPairs, TR>> }
+
+const KernelEntry kTable[] = {
+    LAGKV_PAIR_ENTRY(128, 2, 32), LAGKV_PAIR_ENTRY(128, 2, 16), LAGKV_PAIR_ENTRY(64, 1, 32), LAGKV_PAIR_ENTRY(256, 2, 16),
+};
+}  // namespace
+
+int pair_kernels(const KernelEntry** table) {
+    *table = kTable;
+    return int(sizeof(kTable) / sizeof(kTable[0]));
+}
+}  // namespace lagkv

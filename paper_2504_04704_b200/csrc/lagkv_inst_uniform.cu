@@ -1,0 +1,29 @@
+// Instantiations of the uniform kernel (prefill for short partitions, every append).
+#include "lagkv_tables.h"
+
+namespace lagkv {
+namespace {
+#define LAGKV_ENTRY1(D, V, NW, TR, VAR) \
+    { D, NW, TR, VAR, false, NW * 32, &lagkv_stream_kernel<Geo<D, V, NW, TR>, VAR>, \
+      &smem_total_bytes<Geo<D, V, NW, TR>> }
+#define LAGKV_ENTRY(D, V, NW, TR) LAGKV_ENTRY1(D, V, NW, TR, 0)
+/* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
+#define LAGKV_VARIANT_ENTRIES(D, V) \
+    LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
+
+const KernelEntry kTable[] = {
+    LAGKV_ENTRY(128, 2, 8, 32), LAGKV_ENTRY(128, 2, 4, 32), LAGKV_ENTRY(128, 2, 2, 32),
+    LAGKV_ENTRY(128, 2, 8, 16), LAGKV_ENTRY(128, 2, 4, 16), LAGKV_ENTRY(128, 2, 2, 16),
+    LAGKV_ENTRY(64, 1, 8, 32),  LAGKV_ENTRY(64, 1, 4, 32),  LAGKV_ENTRY(64, 1, 2, 32),
+    LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
+    LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
+    LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+    LAGKV_VARIANT_ENTRIES(128, 2), LAGKV_VARIANT_ENTRIES(64, 1), LAGKV_VARIANT_ENTRIES(256, 2),
+};
+}  // namespace
+
+int uniform_kernels(const KernelEntry** table) {
+    *table = kTable;
+    return int(sizeof(kTable) / sizeof(kTable[0]));
+}
+}  // namespace lagkv
