@@ -165,6 +165,14 @@ def test_prefill_warp_specialised_strided(binding, oracle, layout):
                 tune=dict(warps=12, tile_rows=32, stages=2, ctas_per_sm=1))
 
 
+@pytest.mark.parametrize("L,k", [(4096, 512), (8192, 1024), (8192, 8192), (6000, 7)])
+def test_prefill_longest_partitions(binding, oracle, L, k):
+    """Partitions up to the largest lag the plan accepts (8192): beyond what the warp-specialised
+    kernel holds in shared memory, so the uniform kernel runs, with the selection in registers
+    (L <= 5632 at 256 threads) or in shared memory (radix select)."""
+    run_prefill(binding, oracle, 1, 2, 128, 16 + 3 * L + 77, 16, L, k, seed=L + k)
+
+
 def test_prefill_heavy_outliers(binding, oracle):
     run_prefill(binding, oracle, 1, 8, 128, 16 + 8 * 256 + 200, 16, 256, 32, seed=5, sigma_k=1.5)
 
