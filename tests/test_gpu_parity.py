@@ -177,8 +177,12 @@ def test_prefill_heavy_outliers(binding, oracle):
     run_prefill(binding, oracle, 1, 8, 128, 16 + 8 * 256 + 200, 16, 256, 32, seed=5, sigma_k=1.5)
 
 
-def test_prefill_sink_zero_and_minimal(binding, oracle):
-    run_prefill(binding, oracle, 1, 2, 128, 2 * 128, 0, 128, 32, seed=9)       # n = 2, no sink, no remainder
+@pytest.mark.parametrize("warps", [0, 12, 100])
+def test_prefill_sink_zero_and_minimal(binding, oracle, warps):
+    """n = 2 (one compressed partition), no sink, no remainder, on every kernel family."""
+    tune = dict(warps=warps, tile_rows=32, stages=2, ctas_per_sm=1) if warps else None
+    run_prefill(binding, oracle, 1, 2, 128, 2 * 128, 0, 128, 32, seed=9, tune=tune)
+    run_prefill(binding, oracle, 3, 2, 128, 5 + 2 * 128 + 127, 5, 128, 128, seed=10, tune=tune)   # k = L
 
 
 def test_prefill_identity_when_too_short(binding, oracle):
@@ -220,7 +224,7 @@ def test_zero_range_channel(binding, oracle):
     check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host)
 
 
-@pytest.mark.parametrize("warps", [0, 12])
+@pytest.mark.parametrize("warps", [0, 12, 100])
 def test_indices_only_and_rows_only(binding, oracle, warps):
     B, H, D, sink, L, k = 1, 3, 128, 8, 128, 32
     S = sink + 4 * L + 17
@@ -483,6 +487,15 @@ def test_prefill_equals_incremental_variants(binding, variant):
     assert pos == total and plan.read_status(ws)[0] == 0
     assert seq.tolist() == [one["L_R"]] * B
     assert torch.equal(Kc[:, :, :one["L_R"]], one["K_out"]) and torch.equal(Vc[:, :, :one["L_R"]], one["V_out"])
+
+
+@pytest.mark.parametrize("D", [64, 256])
+def test_append_head_dims(binding, oracle, D):
+    sink, L, k = 8, 96, 24
+    stat = [sink, sink + 3 * k]
+    seq = [stat[0] + 3 * L + 3, stat[1] + 2 * L]
+    r = append_case(binding, oracle, 2, 3, D, seq[0] + 9, sink, L, k, seq, stat, 2, seed=D)
+    check_append(r, 2)
 
 
 def test_append_capacity_error_leaves_sequence_alone(binding, oracle):
