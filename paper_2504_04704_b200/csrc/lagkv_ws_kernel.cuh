@@ -12,8 +12,9 @@
 //     tensor meet once per partition on a named barrier to combine their min / max.
 //   * 3 select warps: softmax over the partition, K + V (Eq. 11) and top-k with ties to
 //     the lower index -- one partition behind the streamers, overlapped with them.  They
-//     publish where the kept rows come from; the rows are moved by the copy warp or, what it
-//     has not claimed by the end, in the gather phase.
+//     publish where the kept rows come from and move the rows of every second partition
+//     themselves; the others are moved by the copy warp or, what it has not claimed by the
+//     end, in the gather phase.
 //   * 1 copy warp: moves rows global -> shared -> global with bulk async copies: the kept
 //     rows of partitions whose positions are published (bandwidth the streamers leave
 //     unused), and the rows that are kept verbatim (sink and sliding window) of ALL units,
@@ -283,19 +284,28 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 score_and_select<kWsSelThreads>(sg0, sg1, L, k, !l2norm, scores_g, kept, sc, etid, sync_sel, [&] {
                     if (etid == 0) mbar_arrive(ebar);
                 });
-                // the kept rows themselves are moved by the copy warp or in the gather phase;
-                // here only their source positions are recorded: in idx_out when the caller
-                // wants it, else in the first word of each destination row of K_out
+                // where the kept rows come from: in idx_out when the caller wants it, else (even
+                // slots only, whose rows the copy warp or the gather phase move later) in the
+                // first word of each destination row of K_out
                 {
                     const long long o = (long long)u * P.L_R + sink + p * k;
                     const int row0 = sink + p * L;
                     if (P.idx_out != nullptr) {
                         for (int j = etid; j < k; j += kWsSelThreads) P.idx_out[o + j] = row0 + kept[j];
-                    } else if (P.K_out != nullptr) {
+                    } else if (P.K_out != nullptr && !(i & 1)) {
                         for (int j = etid; j < k; j += kWsSelThreads)
                             *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::D) = row0 + kept[j];
                     }
                 }
+                // Odd slots: the select warps, idle most of the time, move the kept rows themselves
+                // while kept[] is at hand (even slots are left to the copy warp and the gather
+                // phase).  Every second slot is what they can carry without holding up the
+                // streamers; it takes a fifth of the rows off the gather phase.
+                if ((i & 1) && P.K_out != nullptr)
+                    emit_kept<kWsSelThreads, G::VPR, 16>(unit_base(P.K, u), unit_base(P.V, u), P.ss,
+                                                         P.K_out + (long long)u * P.L_R * G::D,
+                                                         P.V_out + (long long)u * P.L_R * G::D, sink + p * L,
+                                                         sink + p * k, kept, k, nullptr, etid);
                 __threadfence_block();  // the positions above are visible before the count below
                 sync_sel();             // every thread is done with kept[] and has written its share
             } else if (etid == 0) {
@@ -339,10 +349,11 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             const int done = *sel_done;
             if (rows_wanted && !dead) {
                 if (!gclaimed) {
-                    // slots without kept rows (top partitions, the statistics-only extra slot)
+                    // skip slots without kept rows (top partitions, the statistics-only extra slot)
+                    // and the odd slots, whose rows the select warps move
                     while (gslot < nslots) {
                         const long long sl = s_lo + gslot;
-                        if (slot_scored(int(sl % spu)) && sl >= s_first) break;
+                        if (slot_scored(int(sl % spu)) && sl >= s_first && !(gslot & 1)) break;
                         ++gslot;
                     }
                     if (gslot < done && done < nslots) {
@@ -457,7 +468,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         const long long s_from = s_lo + *reinterpret_cast<volatile int*>(&sc.claimed);
         for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
             const int u = int(s / spu), sj = int(s % spu), p = slot_part(sj);
-            if (!slot_scored(sj)) continue;
+            if (!slot_scored(sj) || ((s - s_lo) & 1)) continue;  // odd slots: done by the select warps
             const uint16_t* srcK = unit_base(P.K, u);
             const uint16_t* srcV = unit_base(P.V, u);
             const long long o = (long long)u * P.L_R + sink + p * k;
