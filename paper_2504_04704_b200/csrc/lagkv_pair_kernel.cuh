@@ -12,8 +12,7 @@
 //     and derive the next coefficients themselves: no barrier between streaming warps at all;
 //   * the epilogue warp takes the two sigma vectors (double buffered, mbarrier hand-off), runs
 //     softmax, K + V (Eq. 11) and the top-k entirely with warp shuffles, writes the positions
-//     and copies the kept rows right away -- they were streamed microseconds ago and come
-//     from L2 -- as well as the unit's window and sink rows.
+//     and copies the kept rows right away, as well as the unit's window and sink rows.
 //
 // Scores are bit-identical to the other kernels' (same row sums, same integer softmax
 // denominators, same exp and reciprocal), so the selection is too.
