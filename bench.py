@@ -330,7 +330,7 @@ def main():
                     "is overwritten before each" % (input_bytes / 1e9))},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg,
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": "lagkv_ws_kernel" if info["block"] == 384 else "lagkv_stream_kernel"},
+                     "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": info["kernel"]},
         "clocks": clocks,
         "gpu_launches": args.steps * info["launches"],
     }

@@ -216,9 +216,11 @@ int lagkv_read_status(lagkv_plan_t plan, void *workspace, void *cuda_stream,
 
 /*
  * Launch shape the plan uses for a prefill of S_in rows: info[0] = grid, info[1] = block
- * threads, info[2] = dynamic shared memory bytes, info[3] = kernel launches per call.
+ * threads, info[2] = dynamic shared memory bytes, info[3] = kernel launches per call,
+ * info[4] = kernel family (0 = identity copy, 1 = uniform kernel, 2 = warp-specialised
+ * kernel, 3 = pair kernel), info[5] = reserved (0).
  */
-int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]);
+int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]);
 
 /*
  * Tuning override of the launch shape: warps per CTA (2, 4 or 8 = the uniform kernel, used

@@ -90,7 +90,7 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_read_status.restype = ctypes.c_int
     lib.lagkv_read_status.argtypes = [vp, vp, vp, ctypes.POINTER(i32 * 4)]
     lib.lagkv_launch_info.restype = ctypes.c_int
-    lib.lagkv_launch_info.argtypes = [vp, i64, ctypes.POINTER(i32 * 4)]
+    lib.lagkv_launch_info.argtypes = [vp, i64, ctypes.POINTER(i32 * 6)]
     lib.lagkv_plan_tune.restype = ctypes.c_int
     lib.lagkv_plan_tune.argtypes = [vp, i32, i32, i32, i32]
     lib.lagkv_selftest_bounded_wait.restype = ctypes.c_int
@@ -163,9 +163,10 @@ class Plan:
         return int(self.lib.lagkv_workspace_bytes(self.handle, int(max_new_chunks)))
 
     def launch_info(self, S_in: int) -> dict:
-        info = (ctypes.c_int32 * 4)()
+        info = (ctypes.c_int32 * 6)()
         _check(self.lib.lagkv_launch_info(self.handle, int(S_in), ctypes.byref(info)), "lagkv_launch_info")
-        return {"grid": info[0], "block": info[1], "smem": info[2], "launches": info[3]}
+        kernel = ("lagkv_copy_kernel", "lagkv_stream_kernel", "lagkv_ws_kernel", "lagkv_pair_kernel")[info[4]]
+        return {"grid": info[0], "block": info[1], "smem": info[2], "launches": info[3], "kernel": kernel}
 
     def tune(self, warps=0, tile_rows=0, stages=0, ctas_per_sm=0) -> None:
         _check(self.lib.lagkv_plan_tune(self.handle, int(warps), int(tile_rows), int(stages), int(ctas_per_sm)),

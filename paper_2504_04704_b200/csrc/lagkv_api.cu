@@ -448,7 +448,7 @@ int lagkv_read_status(lagkv_plan_t plan, void* workspace, void* cuda_stream, int
     return host_status[0];
 }
 
-int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
+int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]) {
     if (plan == nullptr || info == nullptr || S_in < 0) return LAGKV_EINVAL;
     const lagkv_config& c = plan->cfg;
     const long long U = (long long)c.B * c.H_kv;
@@ -460,6 +460,7 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
         info[1] = 256;
         info[2] = 0;
         info[3] = S_in > 0 ? 1 : 0;
+        info[4] = info[5] = 0;
         return LAGKV_OK;
     }
     const long long nparts = rest / c.lag;
@@ -471,6 +472,9 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[4]) {
     info[1] = kKernels[shape.kidx].threads;
     info[2] = int(shape.smem);
     info[3] = 1;
+    const KernelEntry& ke = kKernels[shape.kidx];
+    info[4] = !ke.ws ? 1 : (ke.NW == LAGKV_TUNE_PAIRS ? 3 : 2);
+    info[5] = 0;
     return LAGKV_OK;
 }
 
