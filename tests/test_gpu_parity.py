@@ -559,6 +559,68 @@ def test_chunked_prefill_driver_equals_one_shot(binding, oracle):
     np.testing.assert_array_equal(synth.to_bits(drv.V[:, :, :drv.rows]), ref["V_out"])
 
 
+@pytest.mark.parametrize("warps,L,k", [(0, 64, 16), (12, 256, 64), (100, 128, 16), (12, 2048, 256)])
+def test_no_write_outside_the_output_buffers(binding, warps, L, k):
+    """Guard zones before and after every output (rows, indices, scores) and around the
+    workspace stay untouched; the inputs are not modified."""
+    B, H, D, sink = 3, 2, 128, 8
+    S = sink + 5 * L + L // 3
+    K, V = synth.make_kv(B, H, S, D, seed=91, device="cuda:0")
+    K0, V0 = K.clone(), V.clone()
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    if warps:
+        plan.tune(warps=warps, tile_rows=32, stages=2, ctas_per_sm=1)
+    L_R, n_c, G = plan.compressed_len(S), (S - sink) // L - 1, 4096
+
+    def guarded(numel, dtype, fill):
+        buf = torch.full((numel + 2 * G,), fill, dtype=dtype, device="cuda:0")
+        return buf, buf[G:G + numel]
+
+    kb, ko = guarded(B * H * L_R * D, torch.bfloat16, 7.0)
+    vb, vo = guarded(B * H * L_R * D, torch.bfloat16, 7.0)
+    ib, io = guarded(B * H * L_R, torch.int32, -5)
+    sb, so = guarded(B * H * n_c * L, torch.float32, -3.0)
+    wb, wo = guarded(plan.workspace_bytes(), torch.uint8, 0)
+    wb[:G] = 9
+    wb[G + wo.numel():] = 9
+    out = {"K_out": ko.view(B, H, L_R, D), "V_out": vo.view(B, H, L_R, D), "idx": io.view(B, H, L_R),
+           "scores": so.view(B, H, n_c, L)}
+    plan.compress_prefill(K, V, wo, out=out, want_scores=True)
+    assert plan.read_status(wo)[0] == 0
+    for buf, inner, fill in ((kb, ko, 7.0), (vb, vo, 7.0), (ib, io, -5), (sb, so, -3.0), (wb, wo, 9)):
+        assert bool((buf[:G] == fill).all()) and bool((buf[G + inner.numel():] == fill).all())
+    assert torch.equal(K, K0) and torch.equal(V, V0)
+    take = out["idx"].long().unsqueeze(-1).expand(-1, -1, -1, D)
+    assert torch.equal(out["K_out"], torch.gather(K, 2, take)) and torch.equal(out["V_out"], torch.gather(V, 2, take))
+
+
+def test_append_writes_nothing_beyond_the_valid_rows(binding):
+    """In-place append: rows at and beyond the pre-call length, other sequences' skipped caches
+    and guard zones around the length arrays stay untouched."""
+    B, H, D, sink, L, k = 3, 2, 128, 8, 128, 32
+    S_cap = sink + 4 * L
+    K, V = synth.make_kv(B, H, S_cap, D, seed=92, device="cuda:0")
+    K0, V0 = K.clone(), V.clone()
+    lens = torch.full((64,), -9, dtype=torch.int32, device="cuda:0")
+    seq, stat = lens[16:16 + B], lens[40:40 + B]
+    seq.copy_(torch.tensor([sink + 3 * L + 5, sink + 2 * L - 1, sink + 2 * L]))
+    stat.fill_(sink)
+    seq0 = seq.clone()
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace(2)
+    plan.compress_append(K, V, seq, stat, ws, max_new_chunks=2)
+    assert plan.read_status(ws)[0] == 0
+    assert seq.tolist() == [sink + 2 * k + L + 5, sink + 2 * L - 1, sink + k + L]
+    for b in range(B):
+        n0 = int(seq0[b])
+        assert torch.equal(K[b, :, n0:], K0[b, :, n0:]) and torch.equal(V[b, :, n0:], V0[b, :, n0:])
+    assert torch.equal(K[1], K0[1]) and torch.equal(V[1], V0[1])           # the skipped sequence
+    keep = torch.ones(64, dtype=torch.bool, device="cuda:0")
+    keep[16:16 + B] = False
+    keep[40:40 + B] = False
+    assert bool((lens[keep] == -9).all())
+
+
 def test_host_prefill_pipeline_matches_direct_call(binding, oracle):
     """The host end-to-end path (pinned host cache -> device chunks -> compress -> compacted rows
     and indices back on the host, three streams, two staging slots) returns what one direct
