@@ -594,6 +594,43 @@ def test_no_write_outside_the_output_buffers(binding, warps, L, k):
     assert torch.equal(out["K_out"], torch.gather(K, 2, take)) and torch.equal(out["V_out"], torch.gather(V, 2, take))
 
 
+def test_append_state_is_cache_plus_two_lengths(binding):
+    """Checkpoint / resume: the pass keeps no hidden state.  Copying (K, V, seq_len, static_len)
+    after some appends and resuming on the copy with a new plan and workspace gives, bit for
+    bit, what the uninterrupted run gives."""
+    B, H, D, sink, L, k = 2, 2, 128, 4, 64, 16
+    total = sink + 9 * L + 20
+    Ksrc, Vsrc = synth.make_kv(B, H, total, D, seed=93, device="cuda:0")
+
+    def feed(plan, ws, Kc, Vc, seq, stat, lo, hi, step=37):
+        for pos in range(lo, hi, step):
+            t = min(step, hi - pos)
+            s = int(seq[0])
+            Kc[:, :, s:s + t], Vc[:, :, s:s + t] = Ksrc[:, :, pos:pos + t], Vsrc[:, :, pos:pos + t]
+            seq += t
+            plan.compress_append(Kc, Vc, seq, stat, ws, max_new_chunks=1)
+
+    def fresh():
+        plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+        return plan, plan.new_workspace(1)
+
+    Kc = torch.zeros((B, H, sink + 8 * k + 3 * L, D), dtype=torch.bfloat16, device="cuda:0")   # stored rows grow by k per partition
+    Vc = torch.zeros_like(Kc)
+    seq = torch.zeros((B,), dtype=torch.int32, device="cuda:0")
+    stat = torch.full((B,), sink, dtype=torch.int32, device="cuda:0")
+    plan, ws = fresh()
+    half = sink + 4 * L + 11
+    feed(plan, ws, Kc, Vc, seq, stat, 0, half)
+    snap = [t.clone() for t in (Kc, Vc, seq, stat)]
+    feed(plan, ws, Kc, Vc, seq, stat, half, total)
+    plan2, ws2 = fresh()
+    feed(plan2, ws2, *snap, half, total)
+    assert plan.read_status(ws)[0] == 0 and plan2.read_status(ws2)[0] == 0
+    for a, b in zip((Kc, Vc, seq, stat), snap):
+        assert torch.equal(a, b)
+    assert int(stat[0]) == sink + 8 * k
+
+
 def test_append_writes_nothing_beyond_the_valid_rows(binding):
     """In-place append: rows at and beyond the pre-call length, other sequences' skipped caches
     and guard zones around the length arrays stay untouched."""
