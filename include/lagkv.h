@@ -63,7 +63,7 @@ enum lagkv_variant {
 typedef struct {
     int32_t B;          /* sequences (times layers when folded), >= 1                 */
     int32_t H_kv;       /* KV heads per sequence, >= 1; selection is per KV head      */
-    int32_t D;          /* head_dim; supported: 64, 128, 256 (128 is the tuned case)  */
+    int32_t D;          /* head_dim; supported: 64, 96, 128, 256 (128 is tuned)      */
     int32_t sink;       /* S: attention-sink rows kept verbatim, >= 0                 */
     int32_t lag;        /* L: partition size, 2 <= L <= 8192                          */
     double keep_ratio;  /* r in (0, 1]; k = ceil(r*L - 1e-9) clamped to [1, L]        */

@@ -207,7 +207,7 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
     if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
-    if (cfg->D != 64 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
+    if (cfg->D != 64 && cfg->D != 96 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
     if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
 
     lagkv_plan_s* pl = new (std::nothrow) lagkv_plan_s();

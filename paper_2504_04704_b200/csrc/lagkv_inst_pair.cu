@@ -9,6 +9,7 @@ namespace {
 
 const KernelEntry kTable[] = {
     LAGKV_PAIR_ENTRY(128, 2, 32), LAGKV_PAIR_ENTRY(128, 2, 16), LAGKV_PAIR_ENTRY(64, 1, 32), LAGKV_PAIR_ENTRY(256, 2, 16),
+    LAGKV_PAIR_ENTRY(96, 3, 32),
 };
 }  // namespace
 

@@ -18,7 +18,10 @@ const KernelEntry kTable[] = {
     LAGKV_ENTRY(64, 1, 8, 16),  LAGKV_ENTRY(64, 1, 4, 16),  LAGKV_ENTRY(64, 1, 2, 16),
     LAGKV_ENTRY(256, 2, 8, 32), LAGKV_ENTRY(256, 2, 4, 32), LAGKV_ENTRY(256, 2, 2, 32),
     LAGKV_ENTRY(256, 2, 8, 16), LAGKV_ENTRY(256, 2, 4, 16), LAGKV_ENTRY(256, 2, 2, 16),
+    LAGKV_ENTRY(96, 3, 8, 32),  LAGKV_ENTRY(96, 3, 4, 32),  LAGKV_ENTRY(96, 3, 2, 32),
+    LAGKV_ENTRY(96, 3, 8, 16),  LAGKV_ENTRY(96, 3, 4, 16),  LAGKV_ENTRY(96, 3, 2, 16),
     LAGKV_VARIANT_ENTRIES(128, 2), LAGKV_VARIANT_ENTRIES(64, 1), LAGKV_VARIANT_ENTRIES(256, 2),
+    LAGKV_VARIANT_ENTRIES(96, 3),
 };
 }  // namespace
 

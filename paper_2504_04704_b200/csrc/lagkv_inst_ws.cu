@@ -11,7 +11,8 @@ namespace {
 
 const KernelEntry kTable[] = {
     LAGKV_WS_ENTRY(128, 2, 8, 32), LAGKV_WS_ENTRY(128, 2, 8, 16), LAGKV_WS_ENTRY(64, 1, 8, 32),
-    LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16),
+    LAGKV_WS_ENTRY(64, 1, 8, 16), LAGKV_WS_ENTRY(256, 2, 8, 16), LAGKV_WS_ENTRY(96, 3, 8, 32),
+    LAGKV_WS_ENTRY(96, 3, 8, 16),
 };
 }  // namespace
 

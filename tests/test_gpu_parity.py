@@ -12,6 +12,8 @@ Bars:
     fp32 scores -- bit-exact, no tolerance;
   * compacted K/V rows bit-exact given the indices; sink and window bit-identical.
 """
+import functools
+
 import numpy as np
 import pytest
 import torch
@@ -125,10 +127,18 @@ def test_prefill_lag_sweep(binding, oracle, L, k, S_extra):
     run_prefill(binding, oracle, 2, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L)
 
 
-@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("D", [64, 96, 128, 256])
 @pytest.mark.parametrize("ddof", [0, 1])
 def test_prefill_head_dims(binding, oracle, D, ddof):
     run_prefill(binding, oracle, 1, 4, D, 16 + 6 * 128 + 37, 16, 128, 32, seed=D + ddof, ddof=ddof)
+
+
+@pytest.mark.parametrize("D,tile_rows", [(64, 32), (96, 32), (96, 16), (256, 16)])
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_prefill_warp_specialised_head_dims(binding, oracle, D, tile_rows, variant):
+    run = run_l2norm if variant == binding.VARIANT_L2NORM else functools.partial(run_prefill, variant=variant)
+    run(binding, oracle, 2, 3, D, 16 + 5 * 256 + 201, 16, 256, 64, seed=D + tile_rows + variant,
+        tune=dict(warps=12, tile_rows=tile_rows))
 
 
 @pytest.mark.parametrize("layout", ["bshd", "padded"])
@@ -272,7 +282,7 @@ def test_pair_kernel_prefill(binding, oracle, L, k, S_extra, B):
     run_prefill(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 3, tune=PAIRS)
 
 
-@pytest.mark.parametrize("D,tile_rows", [(64, 32), (256, 16), (128, 16)])
+@pytest.mark.parametrize("D,tile_rows", [(64, 32), (96, 32), (256, 16), (128, 16)])
 @pytest.mark.parametrize("ddof", [0, 1])
 def test_pair_kernel_head_dims(binding, oracle, D, tile_rows, ddof):
     run_prefill(binding, oracle, 2, 4, D, 16 + 6 * 128 + 37, 16, 128, 32, seed=D + ddof + 1, ddof=ddof,
@@ -328,11 +338,15 @@ L2_REL_TOL = 1e-5     # |gpu - oracle| <= L2_REL_TOL * |oracle| for the norm sco
                                            (2048, 256, 100, 1), (37, 5, 36, 2)])
 def test_l2norm_prefill(binding, oracle, L, k, S_extra, B):
     """L2-norm variant (Eq. 16): score = -||K row||, no softmax, V only gathered."""
-    H, D, sink = 3, 128, 4
     n = 5 if L >= 512 else 9
-    S = sink + n * L + S_extra
-    K, V = synth.make_kv(B, H, S, D, seed=L + 9, device="cuda:0")
+    run_l2norm(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 9)
+
+
+def run_l2norm(binding, oracle, B, H, D, S, sink, L, k, seed, tune=None):
+    K, V = synth.make_kv(B, H, S, D, seed=seed, device="cuda:0")
     plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=binding.VARIANT_L2NORM, device=0)
+    if tune:
+        plan.tune(**tune)
     ws = plan.new_workspace()
     out = plan.compress_prefill(K, V, ws, want_scores=True)
     assert plan.read_status(ws)[0] == 0
@@ -489,7 +503,7 @@ def test_prefill_equals_incremental_variants(binding, variant):
     assert torch.equal(Kc[:, :, :one["L_R"]], one["K_out"]) and torch.equal(Vc[:, :, :one["L_R"]], one["V_out"])
 
 
-@pytest.mark.parametrize("D", [64, 256])
+@pytest.mark.parametrize("D", [64, 96, 256])
 def test_append_head_dims(binding, oracle, D):
     sink, L, k = 8, 96, 24
     stat = [sink, sink + 3 * k]
@@ -704,7 +718,7 @@ def test_bounded_wait_gives_up_and_reports(binding):
 # ----------------------------------------------------------------------- argument checks
 def test_argument_errors(binding):
     with pytest.raises(binding.LagKVError) as e:
-        binding.Plan(1, 1, 96, 4, 64, device=0)
+        binding.Plan(1, 1, 80, 4, 64, device=0)
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
     with pytest.raises(binding.LagKVError) as e:
         binding.Plan(1, 1, 128, 4, 1, device=0)
