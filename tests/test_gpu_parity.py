@@ -463,6 +463,40 @@ def test_append_multi_chunk(binding, oracle, L, k, chunks):
     check_append(r, 2)
 
 
+def test_ragged_batch_prefill_in_place(binding, oracle):
+    """A batch of prompts of different lengths, compressed in place through the append entry
+    point with static_len = sink: every sequence equals its own one-shot prefill (Eq. 7-12)."""
+    sink, L, k, H, D = 16, 128, 32, 3, 128
+    seq = [sink + 9 * L + 77, sink + 2 * L, sink + 2 * L - 1, sink + 5 * L, 40, sink + 12 * L + 127]
+    B, S_cap = len(seq), max(seq) + 5
+    K, V = synth.make_kv(B, H, S_cap, D, seed=77, device="cuda:0")
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
+    stat_d = torch.full((B,), sink, dtype=torch.int32, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    chunks = max((s - sink) // L - 1 for s in seq)
+    ws = plan.new_workspace(chunks)
+    idx_out = torch.full((B, H, chunks * k), -1, dtype=torch.int32, device="cuda:0")
+    plan.compress_append(K, V, seq_d, stat_d, ws, max_new_chunks=chunks, idx_out=idx_out)
+    assert plan.read_status(ws)[0] == 0
+    Kn, Vn, idx = synth.to_bits(K), synth.to_bits(V), idx_out.cpu().numpy()
+    for b in range(B):
+        ref = oracle.compress(Kb[b:b + 1, :, :seq[b]], Vb[b:b + 1, :, :seq[b]], sink, L, k)
+        L_R, n_c = ref["L_R"], ref["n_c"]
+        assert int(seq_d[b]) == L_R and int(stat_d[b]) == sink + n_c * k
+        mism = 0
+        for h in range(H):
+            got = idx[b, h, :n_c * k]
+            want = ref["idx"][0, h, sink:sink + n_c * k]
+            mism += int((got != want).any())
+            src = np.concatenate([np.arange(sink), got, ref["idx"][0, h, sink + n_c * k:]]).astype(np.int64)
+            np.testing.assert_array_equal(Kn[b, h, :L_R], Kb[b, h, src])
+            np.testing.assert_array_equal(Vn[b, h, :L_R], Vb[b, h, src])
+            assert np.all(idx[b, h, n_c * k:] == -1)
+        assert mism == 0, f"sequence {b}: {mism} heads differ from the one-shot oracle"
+        np.testing.assert_array_equal(Kn[b, :, seq[b]:], Kb[b, :, seq[b]:])
+
+
 @pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("L,k,chunks", [(64, 16, 4), (256, 32, 3), (512, 128, 1)])
 def test_append_variants(binding, oracle, variant, L, k, chunks):
