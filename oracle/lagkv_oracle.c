@@ -7,8 +7,10 @@
  * check the CUDA library; the CUDA library never calls it and shares no code with it.
  *
  * Every step is written in the order the paper's Methodology lists it, one loop per
- * step, with no blocking, fusion or reordering.  Inputs are bf16 bit patterns
- * (uint16_t); each is widened exactly to double before any arithmetic.
+ * step, with no blocking, fusion or reordering.  Inputs are 16-bit patterns
+ * (uint16_t) in the cache's storage format, bf16 (the default) or IEEE fp16; each is
+ * widened exactly to double before any arithmetic.  The paper does not name a storage
+ * format; the method is the same for either.
  *
  * Readings taken where the paper leaves a choice:
  *   - min/max are taken over the tokens of the reference partition, one pair per
@@ -40,6 +42,8 @@
 
 enum { LAGKV_ORACLE_LAGKV = 0, LAGKV_ORACLE_LOCALKV = 1, LAGKV_ORACLE_L2NORM = 2 };
 
+enum { LAGKV_ORACLE_BF16 = 0, LAGKV_ORACLE_FP16 = 1 };
+
 /* bf16 bit pattern -> double, exact (bf16 is the upper half of an IEEE binary32). */
 static double bf16_to_double(uint16_t bits)
 {
@@ -47,6 +51,32 @@ static double bf16_to_double(uint16_t bits)
     float f;
     memcpy(&f, &w, sizeof f);
     return (double)f;
+}
+
+/* IEEE binary16 bit pattern -> double, exact: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double fp16_to_double(uint16_t bits)
+{
+    int sign = bits >> 15, e = (bits >> 10) & 31, frac = bits & 1023;
+    double v;
+    if (e == 0)
+        v = ldexp((double)frac, -24);                 /* zero and subnormals */
+    else if (e == 31)
+        v = frac ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)frac / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+/* The storage format of the cache is the only place a value's bits are interpreted. */
+static double decode(uint16_t bits, int storage)
+{
+    return storage == LAGKV_ORACLE_FP16 ? fp16_to_double(bits) : bf16_to_double(bits);
+}
+
+/* out[i] = value of bits[i] in the given storage format (exposed so that tests can pin it). */
+void lagkv_oracle_decode(const uint16_t *bits, int64_t n, int storage, double *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = decode(bits[i], storage);
 }
 
 int lagkv_oracle_num_threads(void)
@@ -94,11 +124,11 @@ int64_t lagkv_oracle_compressed_len(int64_t seq_len, int64_t static_len, int64_t
 
 /*
  * score(Z) of Eq. 10 for one tensor of one partition.
- *   cur, ref : [L, D] bf16 rows, row_stride elements apart
+ *   cur, ref : [L, D] rows of 16-bit values, row_stride elements apart
  *   out      : [L] softmax(Std(normalised cur))
  */
 static void tensor_score(const uint16_t *cur, const uint16_t *ref, int64_t L, int64_t D,
-                         int64_t row_stride, int ddof, double *out)
+                         int64_t row_stride, int ddof, int storage, double *out)
 {
     double *mn = (double *)malloc(sizeof(double) * (size_t)D);
     double *mx = (double *)malloc(sizeof(double) * (size_t)D);
@@ -107,10 +137,10 @@ static void tensor_score(const uint16_t *cur, const uint16_t *ref, int64_t L, in
 
     /* Eq. 7 and Eq. 8: per channel, min and max over the reference tokens. */
     for (int64_t c = 0; c < D; ++c) {
-        mn[c] = bf16_to_double(ref[c]);
+        mn[c] = decode(ref[c], storage);
         mx[c] = mn[c];
         for (int64_t t = 1; t < L; ++t) {
-            double z = bf16_to_double(ref[t * row_stride + c]);
+            double z = decode(ref[t * row_stride + c], storage);
             if (z < mn[c]) mn[c] = z;
             if (z > mx[c]) mx[c] = z;
         }
@@ -119,7 +149,7 @@ static void tensor_score(const uint16_t *cur, const uint16_t *ref, int64_t L, in
     for (int64_t t = 0; t < L; ++t) {
         /* Eq. 9: min-max normalisation of the current token, channel by channel. */
         for (int64_t c = 0; c < D; ++c) {
-            double z = bf16_to_double(cur[t * row_stride + c]);
+            double z = decode(cur[t * row_stride + c], storage);
             double range = mx[c] - mn[c];
             y[c] = (range > 0.0) ? (z - mn[c]) / range : 0.0;
         }
@@ -160,13 +190,13 @@ static void tensor_score(const uint16_t *cur, const uint16_t *ref, int64_t L, in
 void lagkv_oracle_partition_scores(const uint16_t *Kcur, const uint16_t *Vcur,
                                    const uint16_t *Kref, const uint16_t *Vref, int64_t L,
                                    int64_t D, int64_t row_stride, int ddof, int variant,
-                                   double *score, double *sK, double *sV)
+                                   int storage, double *score, double *sK, double *sV)
 {
     if (variant == LAGKV_ORACLE_L2NORM) {
         for (int64_t t = 0; t < L; ++t) {
             double ss = 0.0;
             for (int64_t c = 0; c < D; ++c) {
-                double z = bf16_to_double(Kcur[t * row_stride + c]);
+                double z = decode(Kcur[t * row_stride + c], storage);
                 ss += z * z;
             }
             score[t] = -sqrt(ss);
@@ -175,8 +205,8 @@ void lagkv_oracle_partition_scores(const uint16_t *Kcur, const uint16_t *Vcur,
     }
     double *a = (double *)malloc(sizeof(double) * (size_t)L);
     double *b = (double *)malloc(sizeof(double) * (size_t)L);
-    tensor_score(Kcur, Kref, L, D, row_stride, ddof, a);
-    tensor_score(Vcur, Vref, L, D, row_stride, ddof, b);
+    tensor_score(Kcur, Kref, L, D, row_stride, ddof, storage, a);
+    tensor_score(Vcur, Vref, L, D, row_stride, ddof, storage, b);
     for (int64_t t = 0; t < L; ++t) score[t] = a[t] + b[t]; /* Eq. 11 */
     if (sK) memcpy(sK, a, sizeof(double) * (size_t)L);
     if (sV) memcpy(sV, b, sizeof(double) * (size_t)L);
@@ -208,7 +238,7 @@ void lagkv_oracle_topk(const double *score, int64_t L, int64_t k, int32_t *idx_o
 }
 
 /*
- * One compress pass over contiguous caches K, V of shape [B, H, seq_len, D] (bf16 bits).
+ * One compress pass over contiguous caches K, V of shape [B, H, seq_len, D] (16-bit patterns).
  * The first static_len rows of every (b, h) are the sink plus the already compressed
  * part and are copied through; the rest is cut into partitions of L rows, partition p
  * is scored against partition p+1, k rows of it are kept, and the last full partition
@@ -222,7 +252,7 @@ void lagkv_oracle_topk(const double *score, int64_t L, int64_t k, int32_t *idx_o
  */
 int64_t lagkv_oracle_compress(const uint16_t *K, const uint16_t *V, int64_t B, int64_t H,
                               int64_t seq_len, int64_t D, int64_t static_len, int64_t L,
-                              int64_t k, int ddof, int variant, int32_t *idx_out,
+                              int64_t k, int ddof, int variant, int storage, int32_t *idx_out,
                               uint16_t *K_out, uint16_t *V_out, double *scores_out)
 {
     int64_t L_R = lagkv_oracle_compressed_len(seq_len, static_len, L, k);
@@ -249,8 +279,8 @@ int64_t lagkv_oracle_compress(const uint16_t *K, const uint16_t *V, int64_t B, i
                 int64_t cur = static_len + p * L;
                 int64_t ref = (variant == LAGKV_ORACLE_LOCALKV) ? cur : cur + L;
                 lagkv_oracle_partition_scores(Ku + cur * D, Vu + cur * D, Ku + ref * D,
-                                              Vu + ref * D, L, D, D, ddof, variant, score,
-                                              NULL, NULL);
+                                              Vu + ref * D, L, D, D, ddof, variant, storage,
+                                              score, NULL, NULL);
                 if (scores_out)
                     memcpy(scores_out + (u * n_c + p) * L, score, sizeof(double) * (size_t)L);
                 lagkv_oracle_topk(score, L, k, keep);

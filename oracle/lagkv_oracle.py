@@ -4,7 +4,8 @@ TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
 benchmark's CPU-baseline leg.  Nothing here is part of the CUDA library, and the CUDA
 library imports nothing from here.
 
-All arrays are numpy; K and V are bf16 bit patterns held as ``uint16`` with shape
+All arrays are numpy; K and V are 16-bit patterns (bf16 by default, fp16 with
+``storage=STORAGE_FP16``) held as ``uint16`` with shape
 ``[B, H, seq_len, D]`` (C-contiguous).  The arithmetic lives in the C file; this
 module only compiles it (gcc, on first use), marshals arguments and implements the
 append bookkeeping of Section 2.2 (bullets 2-4) on top of ``compress``.
@@ -23,6 +24,7 @@ _SRC = _HERE / "lagkv_oracle.c"
 _LIB = _HERE / "liblagkv_oracle.so"
 
 VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
+STORAGE_BF16, STORAGE_FP16 = 0, 1
 
 _lib = None
 
@@ -53,11 +55,13 @@ def _load():
     lib.lagkv_oracle_compressed_len.restype = i64
     lib.lagkv_oracle_compressed_len.argtypes = [i64, i64, i64, i64]
     lib.lagkv_oracle_partition_scores.restype = None
-    lib.lagkv_oracle_partition_scores.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp, vp, vp]
+    lib.lagkv_oracle_partition_scores.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, ci, vp, vp, vp]
     lib.lagkv_oracle_topk.restype = None
     lib.lagkv_oracle_topk.argtypes = [vp, i64, i64, vp]
     lib.lagkv_oracle_compress.restype = i64
-    lib.lagkv_oracle_compress.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, i64, ci, ci, vp, vp, vp, vp]
+    lib.lagkv_oracle_compress.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp]
+    lib.lagkv_oracle_decode.restype = None
+    lib.lagkv_oracle_decode.argtypes = [vp, i64, ci, vp]
     lib.lagkv_oracle_gather.restype = None
     lib.lagkv_oracle_gather.argtypes = [vp, i64, i64, i64, vp, i64, vp]
     _lib = lib
@@ -71,7 +75,7 @@ def _ptr(a):
 def _u16(a) -> np.ndarray:
     a = np.ascontiguousarray(a)
     if a.dtype != np.uint16:
-        raise TypeError("K/V must be bf16 bit patterns as uint16")
+        raise TypeError("K/V must be 16-bit patterns (bf16 or fp16) as uint16")
     return a
 
 
@@ -93,13 +97,22 @@ def compressed_len(seq_len: int, static_len: int, L: int, k: int) -> int:
     return int(_load().lagkv_oracle_compressed_len(int(seq_len), int(static_len), int(L), int(k)))
 
 
-def partition_scores(Kcur, Vcur, Kref, Vref, ddof: int = 1, variant: int = VARIANT_LAGKV):
+def decode(bits, storage: int = STORAGE_BF16) -> np.ndarray:
+    """The float64 value of every 16-bit pattern, as the oracle reads it."""
+    bits = _u16(bits)
+    out = np.zeros(bits.shape, np.float64)
+    _load().lagkv_oracle_decode(_ptr(bits), bits.size, int(storage), _ptr(out))
+    return out
+
+
+def partition_scores(Kcur, Vcur, Kref, Vref, ddof: int = 1, variant: int = VARIANT_LAGKV,
+                     storage: int = STORAGE_BF16):
     """Eq. 7-11 for one partition.  Inputs ``[L, D]`` uint16.  Returns (score, sK, sV)."""
     Kcur, Vcur, Kref, Vref = map(_u16, (Kcur, Vcur, Kref, Vref))
     L, D = Kcur.shape
     score, sK, sV = (np.zeros(L, np.float64) for _ in range(3))
     _load().lagkv_oracle_partition_scores(
-        _ptr(Kcur), _ptr(Vcur), _ptr(Kref), _ptr(Vref), L, D, D, int(ddof), int(variant),
+        _ptr(Kcur), _ptr(Vcur), _ptr(Kref), _ptr(Vref), L, D, D, int(ddof), int(variant), int(storage),
         _ptr(score), _ptr(sK), _ptr(sV))
     return score, sK, sV
 
@@ -113,7 +126,8 @@ def topk(score, k: int) -> np.ndarray:
 
 
 def compress(K, V, static_len: int, L: int, k: int, ddof: int = 1,
-             variant: int = VARIANT_LAGKV, want_rows: bool = True, want_scores: bool = True):
+             variant: int = VARIANT_LAGKV, want_rows: bool = True, want_scores: bool = True,
+             storage: int = STORAGE_BF16):
     """One compress pass (Section 2.2) over ``[B, H, seq_len, D]`` caches.
 
     Returns a dict with ``L_R``, ``idx`` ``[B,H,L_R]`` int32, and optionally ``K_out`` /
@@ -131,7 +145,7 @@ def compress(K, V, static_len: int, L: int, k: int, ddof: int = 1,
     scores = np.zeros((B, H, n_c, L), np.float64) if want_scores else None
     got = _load().lagkv_oracle_compress(
         _ptr(K), _ptr(V), B, H, S, D, int(static_len), int(L), int(k), int(ddof), int(variant),
-        _ptr(idx), _ptr(K_out), _ptr(V_out), _ptr(scores))
+        int(storage), _ptr(idx), _ptr(K_out), _ptr(V_out), _ptr(scores))
     assert got == L_R
     return {"L_R": L_R, "n_c": n_c, "idx": idx, "K_out": K_out, "V_out": V_out, "scores": scores}
 
@@ -148,7 +162,7 @@ def gather(X, idx) -> np.ndarray:
 
 
 def compress_append(K_cache, V_cache, seq_len, static_len, L: int, k: int, ddof: int = 1,
-                    variant: int = VARIANT_LAGKV):
+                    variant: int = VARIANT_LAGKV, storage: int = STORAGE_BF16):
     """Incremental pass on a ``[B, H, S_cap, D]`` cache with per-sequence lengths.
 
     For every sequence b the rows ``[0, static_len[b])`` are the sink plus everything
@@ -169,7 +183,7 @@ def compress_append(K_cache, V_cache, seq_len, static_len, L: int, k: int, ddof:
             kept.append(np.zeros((K_cache.shape[1], 0), np.int32))
             continue
         res = compress(K_cache[b:b + 1, :, :s], V_cache[b:b + 1, :, :s], st, L, k, ddof, variant,
-                       want_scores=False)
+                       want_scores=False, storage=storage)
         L_R, n_c = res["L_R"], res["n_c"]
         K_cache[b, :, :L_R] = res["K_out"][0]
         V_cache[b, :, :L_R] = res["V_out"][0]

@@ -52,8 +52,9 @@ WORKLOADS = {
 
 
 def make_kv(B: int, H: int, S: int, D: int, seed: int, sigma_k: float = 1.0, sigma_v: float = 0.5,
-            rope_theta: float = 500000.0, device="cpu", pos_offset: int = 0):
-    """Return ``(K, V)`` bf16 tensors ``[B, H, S, D]`` on ``device`` (see module docstring)."""
+            rope_theta: float = 500000.0, device="cpu", pos_offset: int = 0, dtype=torch.bfloat16):
+    """Return ``(K, V)`` tensors ``[B, H, S, D]`` of ``dtype`` (bf16, or fp16 for an fp16 cache) on
+    ``device`` (see module docstring); the same fp32 draws are rounded to either format."""
     dev = torch.device(device)
     g = torch.Generator(device=dev)
     g.manual_seed(int(seed))
@@ -69,11 +70,11 @@ def make_kv(B: int, H: int, S: int, D: int, seed: int, sigma_k: float = 1.0, sig
         k[..., :half] = a * cos - b * sin
         k[..., half:] = b * cos + a * sin
         del a, b, cos, sin, ang
-    K = k.to(torch.bfloat16)
+    K = k.to(dtype)
     del k
     v = torch.randn((B, H, S, D), generator=g, device=dev, dtype=torch.float32)
     v *= torch.exp(sigma_v * torch.randn((B, H, S, 1), generator=g, device=dev, dtype=torch.float32))
-    V = v.to(torch.bfloat16)
+    V = v.to(dtype)
     return K, V
 
 
@@ -84,8 +85,8 @@ def make_workload_layer(w: Workload, layer: int, device="cpu", S: int | None = N
 
 
 def to_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> numpy uint16 array of the same shape (bit patterns, on the host)."""
-    assert t.dtype == torch.bfloat16
+    """bf16 (or fp16) tensor -> numpy uint16 array of the same shape (bit patterns, on the host)."""
+    assert t.dtype in (torch.bfloat16, torch.float16)
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 

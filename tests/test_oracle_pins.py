@@ -51,6 +51,59 @@ def small_cache(seed, B=2, H=3, S=4 + 5 * 16 + 7, D=8):
     return rand_bits(rng, (B, H, S, D)), rand_bits(rng, (B, H, S, D))
 
 
+# --------------------------------------------------------------------- storage formats
+def test_decode_every_bit_pattern(oracle):
+    """The oracle's reading of all 65536 patterns: bf16 is the upper half of a binary32,
+    fp16 is IEEE binary16 (held against numpy's float16)."""
+    allbits = np.arange(65536, dtype=np.uint16)
+    with np.errstate(invalid="ignore"):          # signalling NaN patterns
+        want16 = allbits.view(np.float16).astype(np.float64)
+        want_bf = (allbits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    for storage, want in ((oracle.STORAGE_FP16, want16), (oracle.STORAGE_BF16, want_bf)):
+        got = oracle.decode(allbits, storage)
+        assert np.array_equal(np.isnan(got), np.isnan(want))
+        ok = ~np.isnan(want)
+        assert np.array_equal(got[ok], want[ok]) and np.array_equal(np.signbit(got[ok]), np.signbit(want[ok]))
+
+
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_fp16_storage_same_values_same_result(oracle, ddof):
+    """Values that both formats hold exactly give the same scores and picks whichever format
+    stores them, and the fp16 cache agrees with the pure-Python brute force on its values."""
+    rng = np.random.default_rng(5 + ddof)
+    S, L, D, k, n = 3, 8, 4, 3, 4
+    Ls = S + n * L + 5
+    Kf = rng.integers(-64, 65, (1, 1, Ls, D)) / 8.0      # multiples of 1/8 below 8: 7 significant bits
+    Vf = rng.integers(-64, 65, (1, 1, Ls, D)) / 8.0
+    Kb, Vb = bits(Kf), bits(Vf)
+    Kh, Vh = Kf.astype(np.float16).view(np.uint16), Vf.astype(np.float16).view(np.uint16)
+    assert np.array_equal(Kh.view(np.float16).astype(np.float64), Kf)
+    a = oracle.compress(Kb, Vb, S, L, k, ddof=ddof)
+    b = oracle.compress(Kh, Vh, S, L, k, ddof=ddof, storage=oracle.STORAGE_FP16)
+    assert np.array_equal(a["idx"], b["idx"]) and np.array_equal(a["scores"], b["scores"])
+    assert np.array_equal(b["K_out"], np.take_along_axis(Kh, b["idx"][..., None].astype(np.int64), axis=2))
+    assert brute.compress_head(Kf[0, 0].tolist(), Vf[0, 0].tolist(), S, L, k, ddof) == b["idx"][0, 0].tolist()
+
+
+def test_fp16_storage_values_only_fp16_holds(oracle):
+    """Ten fraction bits: values that bf16 cannot hold, scored against numpy on the decoded values."""
+    rng = np.random.default_rng(11)
+    L, D = 16, 8
+    h = (rng.standard_normal((4, L, D)) * 3).astype(np.float16)
+    Kc, Vc, Kr, Vr = (x.view(np.uint16) for x in h)
+    score, sK, sV = oracle.partition_scores(Kc, Vc, Kr, Vr, storage=oracle.STORAGE_FP16)
+    f = h.astype(np.float64)
+    parts = []
+    for cur, ref in ((f[0], f[2]), (f[1], f[3])):
+        y = (cur - ref.min(0)) / (ref.max(0) - ref.min(0))
+        parts.append(scipy.special.softmax(np.std(y, axis=1, ddof=1)))
+    want = parts[0] + parts[1]
+    np.testing.assert_allclose(score, want, rtol=1e-12)
+    np.testing.assert_allclose(sK, parts[0], rtol=1e-12)
+    wrong = oracle.partition_scores(Kc, Vc, Kr, Vr)[0]              # the same bits read as bf16
+    assert not np.allclose(wrong, want, rtol=1e-3)
+
+
 # ------------------------------------------------------------------ worked examples
 @pytest.mark.parametrize("name", ["hand_case_1.txt", "hand_case_2.txt"])
 @pytest.mark.parametrize("ddof", [0, 1])
