@@ -181,6 +181,8 @@ def main():
     ap.add_argument("--tune", default="", help="warps,tile_rows,stages,ctas_per_sm override")
     ap.add_argument("--variant", default="lagkv", choices=["lagkv", "localkv", "l2norm"],
                     help="scoring variant of Section 4.3 (the headline metric is lagkv)")
+    ap.add_argument("--storage", default="bf16", choices=["bf16", "fp16"],
+                    help="storage format of the caches (fp16: device-timed pass only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -213,21 +215,23 @@ def main():
 
     # ---- this rank's cache: all layers folded into the batch dimension, resident in HBM
     Bf = w.layers * w.B
-    K = torch.empty((Bf, w.H, w.S, w.D), dtype=torch.bfloat16, device=dev)
+    store = torch.float16 if args.storage == "fp16" else torch.bfloat16
+    K = torch.empty((Bf, w.H, w.S, w.D), dtype=store, device=dev)
     V = torch.empty_like(K)
     for layer in range(w.layers):
-        k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, shard.rank_seed(w.seed(layer), rank), w.sigma_k, w.sigma_v, device=dev)
+        k_l, v_l = synth.make_kv(w.B, w.H, w.S, w.D, shard.rank_seed(w.seed(layer), rank), w.sigma_k, w.sigma_v,
+                                 device=dev, dtype=store)
         K[layer * w.B:(layer + 1) * w.B], V[layer * w.B:(layer + 1) * w.B] = k_l, v_l
         del k_l, v_l
     variant = {"lagkv": 0, "localkv": 1, "l2norm": 2}[args.variant]
-    plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, variant=variant, device=local)
+    plan = binding.Plan(Bf, w.H, w.D, w.sink, w.lag, keep_ratio=w.ratio, variant=variant, device=local, dtype=store)
     if args.tune:
         t = [int(x) for x in args.tune.split(",")]
         plan.tune(warps=t[0], tile_rows=t[1], stages=t[2], ctas_per_sm=t[3])
     ws = plan.new_workspace()
     L_R = plan.compressed_len(w.S)
-    out = {"K_out": torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, device=dev),
-           "V_out": torch.empty((Bf, w.H, L_R, w.D), dtype=torch.bfloat16, device=dev),
+    out = {"K_out": torch.empty((Bf, w.H, L_R, w.D), dtype=store, device=dev),
+           "V_out": torch.empty((Bf, w.H, L_R, w.D), dtype=store, device=dev),
            "idx": torch.empty((Bf, w.H, L_R), dtype=torch.int32, device=dev)}
     info = plan.launch_info(w.S)
     step = lambda: plan.compress_prefill(K, V, ws, out=out)
@@ -276,7 +280,7 @@ def main():
 
     # ---- end to end: host cache -> device -> compress -> compacted cache back on the host
     e2e = None
-    if not args.no_e2e and variant == 0:
+    if not args.no_e2e and variant == 0 and args.storage == "bf16":
         chunk = max(1, min(4, w.layers)) * w.B
         while Bf % chunk:
             chunk -= 1
@@ -322,7 +326,7 @@ def main():
         "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
                    "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio, "keep_k": plan.k, "L_R": L_R,
                    "variant": args.variant,
-                   "storage": "bf16", "parallelism": f"dp{world} (independent caches per rank, no collective)",
+                   "storage": args.storage, "parallelism": f"dp{world} (independent caches per rank, no collective)",
                    "launch": info,
                    "l2": ("inputs (%.2f GB per rank) are far larger than the 126 MB L2; no flush" % (input_bytes / 1e9))
                    if not flush_l2 else
@@ -336,7 +340,7 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
-    if not args.no_cpu and world == 1 and variant == 0:
+    if not args.no_cpu and world == 1 and variant == 0 and args.storage == "bf16":
         layers_bits = [(synth.to_bits(K[l * w.B:(l + 1) * w.B]), synth.to_bits(V[l * w.B:(l + 1) * w.B]))
                        for l in range(min(4, w.layers))]
         del K, V

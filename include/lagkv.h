@@ -12,7 +12,8 @@
  * rows stay as a sliding window.  The resulting length is Eq. 12.
  *
  * Conventions shared by every entry point
- *   - All cache pointers are DEVICE pointers to bf16 data, 16-byte aligned; scalars and
+ *   - All cache pointers are DEVICE pointers to 16-bit data (bf16, or fp16 when the plan
+ *     says so: "bf16" below stands for the plan's format), 16-byte aligned; scalars and
  *     the config struct are host values.  The library allocates no device memory and
  *     never synchronises the stream, except in lagkv_read_status().
  *   - A cache is addressed as  base + b*stride_b + h*stride_h + s*stride_s + d  (strides
@@ -60,6 +61,11 @@ enum lagkv_variant {
                                   gathered                                             */
 };
 
+enum lagkv_dtype {
+    LAGKV_DTYPE_BF16 = 0, /* the default (a zeroed field)                                */
+    LAGKV_DTYPE_FP16 = 1  /* IEEE binary16 caches; compiled for head_dim 128             */
+};
+
 typedef struct {
     int32_t B;          /* sequences (times layers when folded), >= 1                 */
     int32_t H_kv;       /* KV heads per sequence, >= 1; selection is per KV head      */
@@ -74,6 +80,9 @@ typedef struct {
     int64_t stride_h;
     int64_t stride_s;
     int32_t device;     /* CUDA device ordinal the plan launches on                   */
+    int32_t dtype;      /* enum lagkv_dtype: storage format of every cache of the plan;
+                           the paper names none, and the arithmetic after the exact
+                           widening to fp32 is the same                               */
 } lagkv_config;
 
 /*

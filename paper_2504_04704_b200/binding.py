@@ -47,7 +47,7 @@ class lagkv_config(ctypes.Structure):
         ("keep_ratio", ctypes.c_double),
         ("keep_k", ctypes.c_int32), ("std_ddof", ctypes.c_int32), ("variant", ctypes.c_int32),
         ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_s", ctypes.c_int64),
-        ("device", ctypes.c_int32),
+        ("device", ctypes.c_int32), ("dtype", ctypes.c_int32),
     ]
 
 
@@ -128,16 +128,23 @@ def lagkv_keep_for_target(Ls: int, sink: int, lag: int, target_C: float) -> int:
     return int(load_library().lagkv_keep_for_target(int(Ls), int(sink), int(lag), float(target_C)))
 
 
+DTYPE_BF16, DTYPE_FP16 = 0, 1
+_DTYPES = {torch.bfloat16: DTYPE_BF16, torch.float16: DTYPE_FP16}
+
+
 class Plan:
     """Owns a ``lagkv_plan_t``.  ``device=-1`` makes a host-only plan (integers and launch
     shapes only; it cannot launch)."""
 
     def __init__(self, B, H_kv, D, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1,
-                 variant=VARIANT_LAGKV, strides=(0, 0, 0), device=0):
+                 variant=VARIANT_LAGKV, strides=(0, 0, 0), device=0, dtype=torch.bfloat16):
         lib = load_library()
+        if dtype not in _DTYPES:
+            raise TypeError("dtype must be torch.bfloat16 or torch.float16")
+        self.dtype = dtype
         self.cfg = lagkv_config(int(B), int(H_kv), int(D), int(sink), int(lag), float(keep_ratio), int(keep_k),
                                 int(std_ddof), int(variant), int(strides[0]), int(strides[1]), int(strides[2]),
-                                int(device))
+                                int(device), _DTYPES[dtype])
         self.handle = ctypes.c_void_p()
         _check(lib.lagkv_plan(ctypes.byref(self.cfg), ctypes.byref(self.handle)), "lagkv_plan")
         self.lib = lib
@@ -195,8 +202,8 @@ class Plan:
                                                     _stream(self._dev())), "lagkv_selftest_bounded_wait")
 
     def _check_cache(self, t: torch.Tensor, name: str):
-        if t.dtype != torch.bfloat16 or not t.is_cuda or t.device.index != self.device:
-            raise TypeError(f"{name} must be a bf16 CUDA tensor on device {self.device}")
+        if t.dtype != self.dtype or not t.is_cuda or t.device.index != self.device:
+            raise TypeError(f"{name} must be a {self.dtype} CUDA tensor on device {self.device}")
 
     def compress_prefill(self, K, V, workspace, S_in=None, want_rows=True, want_idx=True, want_scores=False,
                          out=None):
@@ -213,8 +220,8 @@ class Plan:
         dev = self._dev()
         out = dict(out or {})
         if want_rows:
-            out.setdefault("K_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=torch.bfloat16, device=dev))
-            out.setdefault("V_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=torch.bfloat16, device=dev))
+            out.setdefault("K_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=self.dtype, device=dev))
+            out.setdefault("V_out", torch.empty((c.B, c.H_kv, L_R, c.D), dtype=self.dtype, device=dev))
         if want_idx:
             out.setdefault("idx", torch.empty((c.B, c.H_kv, L_R), dtype=torch.int32, device=dev))
         if want_scores:
@@ -267,7 +274,7 @@ class Plan:
             raise TypeError("idx must be a contiguous int32 CUDA tensor")
         n_idx = int(idx.shape[-1])
         S_in = int(K.shape[2] if S_in is None else S_in)
-        K_out = torch.empty((c.B, c.H_kv, n_idx, c.D), dtype=torch.bfloat16, device=dev)
+        K_out = torch.empty((c.B, c.H_kv, n_idx, c.D), dtype=self.dtype, device=dev)
         V_out = None if V is None else torch.empty_like(K_out)
         rc = self.lib.lagkv_gather(self.handle, _ptr(K), _ptr(V), S_in, _ptr(idx), n_idx, _ptr(K_out), _ptr(V_out),
                                    _ptr(workspace), _stream(dev))

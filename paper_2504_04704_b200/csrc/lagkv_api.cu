@@ -18,16 +18,17 @@ namespace {
 
 // every compiled kernel: the three tables live in translation units of their own
 struct KernelTable {
-    const KernelEntry* e[160];
+    static constexpr int kMaxEntries = 256;
+    const KernelEntry* e[kMaxEntries];
     int n = 0;
     KernelTable() {
         const KernelEntry* t;
         int c = uniform_kernels(&t);
-        for (int i = 0; i < c; ++i) e[n++] = t + i;
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = ws_kernels(&t);
-        for (int i = 0; i < c; ++i) e[n++] = t + i;
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = pair_kernels(&t);
-        for (int i = 0; i < c; ++i) e[n++] = t + i;
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
     }
 };
 const KernelTable& table() {
@@ -40,9 +41,10 @@ struct KernelRef {  // kKernels[i] reads like an array
 const KernelRef kKernels;
 #define kNumKernels (table().n)
 
-int find_kernel(int D, int NW, int TR, int variant) {
+int find_kernel(int D, int NW, int TR, int variant, int dtype) {
     for (int i = 0; i < kNumKernels; ++i)
-        if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR && kKernels[i].variant == variant)
+        if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR && kKernels[i].variant == variant &&
+            kKernels[i].dtype == dtype)
             return i;
     return -1;
 }
@@ -94,7 +96,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // Try one launch shape (NW = warps per CTA, 12 = the warp-specialised kernel).
 int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Shape* out) {
-    const int kidx = find_kernel(pl->cfg.D, NW, TR, pl->cfg.variant);
+    const int kidx = find_kernel(pl->cfg.D, NW, TR, pl->cfg.variant, pl->cfg.dtype);
     if (kidx < 0 || stages < 2 || stages > 8 || ctas < 1) return LAGKV_EUNSUPPORTED;
     if (kKernels[kidx].ws && ctas != 1) return LAGKV_EUNSUPPORTED;
     if (NW == LAGKV_TUNE_PAIRS && pl->cfg.lag > 512) return LAGKV_EUNSUPPORTED;  // one warp selects: L <= 512
@@ -207,6 +209,7 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
     if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
+    if (cfg->dtype != LAGKV_DTYPE_BF16 && cfg->dtype != LAGKV_DTYPE_FP16) return LAGKV_EINVAL;
     if (cfg->D != 64 && cfg->D != 96 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
     if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
 

@@ -138,16 +138,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
     return false;
 }
-__device__ __forceinline__ uint32_t bf2_min(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
 // packed pair of fp32 in one 64-bit register (Blackwell f32x2 arithmetic)
 typedef unsigned long long f32x2;
 __device__ __forceinline__ f32x2 pack2(float lo, float hi) {
@@ -168,12 +158,56 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-// two bf16 in one word -> two fp32 (exact)
-__device__ __forceinline__ f32x2 bf2_to_f32x2(uint32_t w) {
-    return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+// Storage format of the cache elements (enum lagkv_dtype): how two packed 16-bit values
+// are compared and widened to fp32.  Both widenings are exact; everything after them is
+// the same fp32 arithmetic.
+template <int DT>
+struct Elem;
+template <>
+struct Elem<0> {  // bf16: the upper half of an IEEE binary32
+    static constexpr uint32_t kPosInf2 = 0x7f807f80u, kNegInf2 = 0xff80ff80u;
+    static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+    static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+};
+template <>
+struct Elem<1> {  // fp16: IEEE binary16
+    static constexpr uint32_t kPosInf2 = 0x7c007c00u, kNegInf2 = 0xfc00fc00u;
+    static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("min.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ float lo(uint32_t w) {
+        float f;
+        asm("{ .reg .b16 l, h; mov.b32 {l, h}, %1; cvt.f32.f16 %0, l; }" : "=f"(f) : "r"(w));
+        return f;
+    }
+    static __device__ __forceinline__ float hi(uint32_t w) {
+        float f;
+        asm("{ .reg .b16 l, h; mov.b32 {l, h}, %1; cvt.f32.f16 %0, h; }" : "=f"(f) : "r"(w));
+        return f;
+    }
+};
+// two packed 16-bit values in one word -> two fp32 (exact)
+template <class E>
+__device__ __forceinline__ f32x2 widen2(uint32_t w) {
+    return pack2(E::lo(w), E::hi(w));
 }
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 __device__ __forceinline__ uint4 ld_nc(const uint4* p) { return __ldg(p); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
@@ -189,8 +223,10 @@ __device__ __forceinline__ uint32_t float_key(float f) {
 }
 
 // ------------------------------------------------------------------------- geometry / smem
-template <int D_, int V_, int NW_, int TR_>
+template <int D_, int V_, int NW_, int TR_, int DT_ = 0>
 struct Geo {
+    using E = Elem<DT_>;                   // storage format of the cache elements
+    static constexpr int DT = DT_;
     static constexpr int D = D_;           // head_dim
     static constexpr int V = V_;           // 16-byte vectors per thread per row
     static constexpr int NW = NW_;         // warps per CTA (even: K warps, odd: V warps)
@@ -281,11 +317,11 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
             for (int c = 0; c < 4; ++c) {
                 const int j = v * 4 + c;
                 if (valid) {
-                    mn[j] = bf2_min(mn[j], w[c]);
-                    mx[j] = bf2_max(mx[j], w[c]);
+                    mn[j] = G::E::min2(mn[j], w[c]);
+                    mx[j] = G::E::max2(mx[j], w[c]);
                 }
                 if (SCORE) {
-                    const f32x2 y = fma2(bf2_to_f32x2(w[c]), a2[j], b2[j]);  // Eq. 9 (centred)
+                    const f32x2 y = fma2(widen2<typename G::E>(w[c]), a2[j], b2[j]);  // Eq. 9 (centred)
                     s1 = add2(s1, y);
                     s2 = fma2(y, y, s2);
                 }
@@ -329,7 +365,7 @@ __device__ __forceinline__ void process_tile_l2(const uint4* __restrict__ tile, 
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const f32x2 z = bf2_to_f32x2(w[c]);
+                const f32x2 z = widen2<typename G::E>(w[c]);
                 s2 = fma2(z, z, s2);
             }
         }
@@ -357,29 +393,29 @@ __device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw
     uint32_t fmn[G::NWORD], fmx[G::NWORD];
 #pragma unroll
     for (int j = 0; j < G::NWORD; ++j) {
-        fmn[j] = 0x7f807f80u;
-        fmx[j] = 0xff80ff80u;
+        fmn[j] = G::E::kPosInf2;
+        fmx[j] = G::E::kNegInf2;
     }
     for (int w = 0; w < nw; ++w) {
         const uint4* st = reinterpret_cast<const uint4*>(stats_t + w * 2 * STAT);
 #pragma unroll
         for (int v = 0; v < G::V; ++v) {
             const uint4 lo = st[v * G::LPR + cg], hi = st[STAT / 4 + v * G::LPR + cg];
-            fmn[v * 4 + 0] = bf2_min(fmn[v * 4 + 0], lo.x);
-            fmn[v * 4 + 1] = bf2_min(fmn[v * 4 + 1], lo.y);
-            fmn[v * 4 + 2] = bf2_min(fmn[v * 4 + 2], lo.z);
-            fmn[v * 4 + 3] = bf2_min(fmn[v * 4 + 3], lo.w);
-            fmx[v * 4 + 0] = bf2_max(fmx[v * 4 + 0], hi.x);
-            fmx[v * 4 + 1] = bf2_max(fmx[v * 4 + 1], hi.y);
-            fmx[v * 4 + 2] = bf2_max(fmx[v * 4 + 2], hi.z);
-            fmx[v * 4 + 3] = bf2_max(fmx[v * 4 + 3], hi.w);
+            fmn[v * 4 + 0] = G::E::min2(fmn[v * 4 + 0], lo.x);
+            fmn[v * 4 + 1] = G::E::min2(fmn[v * 4 + 1], lo.y);
+            fmn[v * 4 + 2] = G::E::min2(fmn[v * 4 + 2], lo.z);
+            fmn[v * 4 + 3] = G::E::min2(fmn[v * 4 + 3], lo.w);
+            fmx[v * 4 + 0] = G::E::max2(fmx[v * 4 + 0], hi.x);
+            fmx[v * 4 + 1] = G::E::max2(fmx[v * 4 + 1], hi.y);
+            fmx[v * 4 + 2] = G::E::max2(fmx[v * 4 + 2], hi.z);
+            fmx[v * 4 + 3] = G::E::max2(fmx[v * 4 + 3], hi.w);
         }
     }
     int zero_range = 0;
 #pragma unroll
     for (int j = 0; j < G::NWORD; ++j) {
-        const float lo0 = bf_lo(fmn[j]), lo1 = bf_hi(fmn[j]);
-        const float hi0 = bf_lo(fmx[j]), hi1 = bf_hi(fmx[j]);
+        const float lo0 = G::E::lo(fmn[j]), lo1 = G::E::hi(fmn[j]);
+        const float hi0 = G::E::lo(fmx[j]), hi1 = G::E::hi(fmx[j]);
         const float r0 = hi0 - lo0, r1 = hi1 - lo1;
         float i0, i1;
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(i0) : "f"(r0));
@@ -1009,8 +1045,8 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         uint32_t mn[G::NWORD], mx[G::NWORD];
 #pragma unroll
         for (int j = 0; j < G::NWORD; ++j) {
-            mn[j] = 0x7f807f80u;  // +inf, +inf
-            mx[j] = 0xff80ff80u;  // -inf, -inf
+            mn[j] = G::E::kPosInf2;  // +inf, +inf
+            mx[j] = G::E::kNegInf2;  // -inf, -inf
         }
         float* sig = tensor ? sg1 : sg0;
 
@@ -1052,8 +1088,8 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         for (int j = 0; j < G::NWORD; ++j) {
 #pragma unroll
             for (int o = G::LPR; o < 32; o <<= 1) {
-                mn[j] = bf2_min(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
-                mx[j] = bf2_max(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+                mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
+                mx[j] = G::E::max2(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
             }
         }
         if (rl == 0) {

@@ -15,6 +15,7 @@ typedef size_t (*smem_fn_t)(int, int);
 struct KernelEntry {
     int D, NW, TR;  // NW: warps per CTA as named in lagkv_plan_tune() (LAGKV_TUNE_PAIRS for the pair kernel)
     int variant;    // enum lagkv_variant the kernel was compiled for
+    int dtype;      // enum lagkv_dtype of the cache elements
     bool ws;        // a persistent prefill-only kernel (warp-specialised or pair), one CTA per SM
     int threads;    // CTA size
     stream_kernel_t fn;

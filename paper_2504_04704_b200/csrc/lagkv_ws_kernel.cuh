@@ -190,8 +190,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             uint32_t mn[G::NWORD], mx[G::NWORD];
 #pragma unroll
             for (int j = 0; j < G::NWORD; ++j) {
-                mn[j] = 0x7f807f80u;  // +inf, +inf
-                mx[j] = 0xff80ff80u;  // -inf, -inf
+                mn[j] = G::E::kPosInf2;  // +inf, +inf
+                mx[j] = G::E::kNegInf2;  // -inf, -inf
             }
             float* sig = sgbase + (buf * 2 + tensor) * Lp;
 
@@ -229,8 +229,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             for (int j = 0; j < G::NWORD; ++j) {
 #pragma unroll
                 for (int o = G::LPR; o < 32; o <<= 1) {
-                    mn[j] = bf2_min(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
-                    mx[j] = bf2_max(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+                    mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
+                    mx[j] = G::E::max2(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
                 }
             }
             uint32_t* stats_t = stats + ((buf * 2 + tensor) * G::WT) * 2 * STAT_WORDS;

@@ -33,9 +33,9 @@ def binding():
     return b
 
 
-def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, variant=0):
+def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, variant=0, storage=0):
     """Compare a GPU prefill result ``out`` (numpy arrays) with the oracle on bit patterns."""
-    ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof, variant=variant)
+    ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof, variant=variant, storage=storage)
     B, H, S, D = Kb.shape
     assert out["L_R"] == ref["L_R"]
     n_c = ref["n_c"]
@@ -86,8 +86,8 @@ def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, vari
 
 
 def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=None, sigma_k=1.0, layout="bhsd",
-                variant=0):
-    K, V = synth.make_kv(B, H, S, D, seed=seed, sigma_k=sigma_k, device="cuda:0")
+                variant=0, dtype=torch.bfloat16):
+    K, V = synth.make_kv(B, H, S, D, seed=seed, sigma_k=sigma_k, device="cuda:0", dtype=dtype)
     strides = (0, 0, 0)
     Kd, Vd = K, V
     if layout == "bshd":        # cache stored [B, S, H, D]; passed as a strided [B, H, S, D] view
@@ -95,12 +95,13 @@ def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=No
         Vd = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
         strides = (S * H * D, D, H * D)
     elif layout == "padded":    # rows padded to D + 8 elements
-        Kp = torch.zeros((B, H, S, D + 8), dtype=torch.bfloat16, device="cuda:0")
+        Kp = torch.zeros((B, H, S, D + 8), dtype=dtype, device="cuda:0")
         Vp = torch.zeros_like(Kp)
         Kp[..., :D], Vp[..., :D] = K, V
         Kd, Vd = Kp, Vp
         strides = (H * S * (D + 8), S * (D + 8), D + 8)
-    plan = binding.Plan(B, H, D, sink, L, keep_k=k, std_ddof=ddof, strides=strides, variant=variant, device=0)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, std_ddof=ddof, strides=strides, variant=variant, device=0,
+                        dtype=dtype)
     if tune:
         plan.tune(**tune)
     ws = plan.new_workspace()
@@ -109,7 +110,8 @@ def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=No
     assert st[0] == 0, f"device status {st}"
     host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
             "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
-    return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host, variant=variant)
+    return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host, variant=variant,
+                                storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
 
 
 # ------------------------------------------------------------------------------- prefill
@@ -342,16 +344,17 @@ def test_l2norm_prefill(binding, oracle, L, k, S_extra, B):
     run_l2norm(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 9)
 
 
-def run_l2norm(binding, oracle, B, H, D, S, sink, L, k, seed, tune=None):
-    K, V = synth.make_kv(B, H, S, D, seed=seed, device="cuda:0")
-    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=binding.VARIANT_L2NORM, device=0)
+def run_l2norm(binding, oracle, B, H, D, S, sink, L, k, seed, tune=None, dtype=torch.bfloat16):
+    K, V = synth.make_kv(B, H, S, D, seed=seed, device="cuda:0", dtype=dtype)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=binding.VARIANT_L2NORM, device=0, dtype=dtype)
     if tune:
         plan.tune(**tune)
     ws = plan.new_workspace()
     out = plan.compress_prefill(K, V, ws, want_scores=True)
     assert plan.read_status(ws)[0] == 0
     Kb, Vb = synth.to_bits(K), synth.to_bits(V)
-    ref = oracle.compress(Kb, Vb, sink, L, k, variant=oracle.VARIANT_L2NORM)
+    ref = oracle.compress(Kb, Vb, sink, L, k, variant=oracle.VARIANT_L2NORM,
+                          storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
     idx = out["idx"].cpu().numpy()
     n_c = ref["n_c"]
     assert out["L_R"] == ref["L_R"]
@@ -385,6 +388,71 @@ def test_variant_shapes(binding):
     assert e.value.code == binding.LAGKV_EUNSUPPORTED
 
 
+# ------------------------------------------------------------------------------ fp16 caches
+FP16_SHAPES = [(64, 16, 60, None), (128, 16, 100, "pairs"), (100, 25, 7, None), (256, 64, 255, None),
+               (512, 128, 3, dict(warps=12, tile_rows=16)), (1024, 256, 1008, None), (2048, 256, 100, None),
+               (1024, 128, 5, dict(warps=8, tile_rows=32))]
+
+
+@pytest.mark.parametrize("L,k,S_extra,tune", FP16_SHAPES)
+def test_fp16_prefill(binding, oracle, L, k, S_extra, tune):
+    """IEEE fp16 caches through every kernel family, against the oracle reading the same bits as fp16."""
+    tune = PAIRS if tune == "pairs" else tune
+    B = 30 if tune is PAIRS else 2
+    n = 5 if L >= 512 else 9
+    run_prefill(binding, oracle, B, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 21, tune=tune, dtype=torch.float16)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("L,k", [(64, 16), (512, 128)])
+def test_fp16_variants(binding, oracle, variant, L, k):
+    if variant == binding.VARIANT_L2NORM:
+        run_l2norm(binding, oracle, 2, 3, 128, 4 + 6 * L + 9, 4, L, k, seed=L + variant, dtype=torch.float16)
+    else:
+        run_prefill(binding, oracle, 2, 3, 128, 4 + 6 * L + 9, 4, L, k, seed=L + variant, variant=variant,
+                    dtype=torch.float16)
+
+
+def test_fp16_append_and_layouts(binding, oracle):
+    sink, L, k = 8, 96, 24
+    stat = [sink, sink + 3 * k]
+    seq = [stat[0] + 3 * L + 3, stat[1] + 2 * L]
+    check_append(append_case(binding, oracle, 2, 3, 128, seq[0] + 9, sink, L, k, seq, stat, 2, seed=5,
+                             dtype=torch.float16), 2)
+    run_prefill(binding, oracle, 2, 4, 128, 40 + 4 * 300 + 111, 40, 300, 75, seed=4, layout="bshd", dtype=torch.float16)
+
+
+def test_fp16_and_bf16_agree_on_values_both_hold(binding):
+    """Values with at most 8 significant bits inside fp16's range: the two storage formats feed
+    the same fp32 values into the same arithmetic, so scores and picks are bit-identical."""
+    B, H, D, sink, L, k = 2, 3, 128, 4, 256, 64
+    S = sink + 6 * L + 77
+    K, V = synth.make_kv(B, H, S, D, seed=91, device="cuda:0")          # bf16: 8 significant bits
+    K, V = K.clamp(-60000, 60000), V.clamp(-60000, 60000)
+    K[K.abs() < 6.2e-5] = 0                                              # below fp16's normal range
+    V[V.abs() < 6.2e-5] = 0
+    Kh, Vh = K.to(torch.float16), V.to(torch.float16)
+    assert torch.equal(Kh.float(), K.float()) and torch.equal(Vh.float(), V.float())
+    res = []
+    for dt, k_, v_ in ((torch.bfloat16, K, V), (torch.float16, Kh, Vh)):
+        plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0, dtype=dt)
+        ws = plan.new_workspace()
+        res.append(plan.compress_prefill(k_, v_, ws, want_scores=True))
+        assert plan.read_status(ws)[0] == 0
+    assert torch.equal(res[0]["idx"], res[1]["idx"]) and torch.equal(res[0]["scores"], res[1]["scores"])
+    assert torch.equal(res[0]["K_out"].float(), res[1]["K_out"].float())
+
+
+def test_fp16_shapes_refused(binding):
+    with pytest.raises(binding.LagKVError) as e:
+        binding.Plan(1, 2, 64, 4, 64, device=0, dtype=torch.float16)       # fp16 is compiled for head_dim 128
+    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+    plan = binding.Plan(1, 2, 128, 4, 64, device=0, dtype=torch.float16)
+    K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
+    with pytest.raises(TypeError):
+        plan.compress_prefill(K, V, plan.new_workspace())                  # a bf16 tensor for an fp16 plan
+
+
 # -------------------------------------------------------------------------------- gather
 def test_gather(binding, oracle):
     B, H, D, S = 2, 3, 128, 500
@@ -407,19 +475,21 @@ def test_gather(binding, oracle):
 
 # -------------------------------------------------------------------------------- append
 def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chunks, seed, tune=None, give_idx=True,
-                variant=0):
-    K, V = synth.make_kv(B, H, S_cap, D, seed=seed, device="cuda:0")
+                variant=0, dtype=torch.bfloat16):
+    K, V = synth.make_kv(B, H, S_cap, D, seed=seed, device="cuda:0", dtype=dtype)
     Kb, Vb = synth.to_bits(K), synth.to_bits(V)
     seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
     stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
-    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0, dtype=dtype)
     if tune:
         plan.tune(**tune)
     ws = plan.new_workspace(max_chunks)
     idx_out = torch.full((B, H, max_chunks * k), -1, dtype=torch.int32, device="cuda:0") if give_idx else None
     plan.compress_append(K, V, seq_d, stat_d, ws, max_new_chunks=max_chunks, idx_out=idx_out)
     st = plan.read_status(ws)
-    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k, variant=variant)
+    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(
+        Kb, Vb, np.array(seq), np.array(stat), L, k, variant=variant,
+        storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
     return dict(K=synth.to_bits(K), V=synth.to_bits(V), seq=seq_d.cpu().numpy(), stat=stat_d.cpu().numpy(),
                 idx=None if idx_out is None else idx_out.cpu().numpy(), status=st,
                 Kr=Kr, Vr=Vr, seq_r=seq_r, stat_r=stat_r, kept=kept, K0=Kb, V0=Vb)
