@@ -150,7 +150,9 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void *K, const void *V, int6
  * oldest partitions are scored against their successors, their k kept rows are packed
  * behind the static part, the window (last full partition + remainder) is moved down
  * behind them, and the call sets static_len += (n-1)*k, seq_len = static_len + L + rem.
- * Other sequences are left untouched (decided on the device: no host sync).
+ * Other sequences are left untouched (decided on the device: no host sync).  The call is
+ * always the same single launch with the same arguments, so it may be captured into a CUDA
+ * graph once and replayed after every decoded token.
  *   max_new_chunks  capacity: a sequence with n-1 > max_new_chunks is left untouched and
  *                   LAGKV_ECAPACITY is recorded in the status block.
  *   idx_out     [B, H, max_new_chunks*k] int32 or NULL: pre-call positions of the rows

@@ -567,6 +567,52 @@ def test_ragged_batch_prefill_in_place(binding, oracle):
         np.testing.assert_array_equal(Kn[b, :, seq[b]:], Kb[b, :, seq[b]:])
 
 
+def test_append_replays_from_a_cuda_graph(binding, oracle):
+    """Decode loop: one captured launch, replayed after every appended token.  Which sequences
+    compress is decided on the device from the lengths, so the graph never changes; the caches
+    and lengths follow the oracle's token-by-token bookkeeping exactly."""
+    B, H, D, sink, L, k, steps = 3, 2, 128, 8, 64, 16, 150
+    S_cap = sink + 3 * L + 8
+    seq0 = [sink + L + 5, sink + 2 * L - 1, 10]
+    fresh_K, fresh_V = synth.make_kv(B, H, steps, D, seed=401, device="cuda:0")
+    K, V = synth.make_kv(B, H, S_cap, D, seed=400, device="cuda:0")
+    Kc, Vc = synth.to_bits(K), synth.to_bits(V)
+    fK, fV = synth.to_bits(fresh_K), synth.to_bits(fresh_V)
+    seq_ref, stat_ref = np.array(seq0, dtype=np.int64), np.full(B, sink, dtype=np.int64)
+    seq = torch.tensor(seq0, dtype=torch.int32, device="cuda:0")
+    stat = torch.full((B,), sink, dtype=torch.int32, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace(1)
+    bidx = torch.arange(B, device="cuda:0")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        plan.compress_append(K, V, seq, stat, ws, max_new_chunks=1)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(synth.to_bits(K), Kc)             # capturing ran nothing
+    triggers = 0
+    for t in range(steps):
+        K[bidx, :, seq.long()] = fresh_K[:, :, t]                   # the model writes one new row per sequence
+        V[bidx, :, seq.long()] = fresh_V[:, :, t]
+        seq += 1
+        graph.replay()
+        for b in range(B):
+            Kc[b, :, seq_ref[b]], Vc[b, :, seq_ref[b]] = fK[b, :, t], fV[b, :, t]
+        seq_ref += 1
+        triggers += int(((seq_ref - stat_ref) >= 2 * L).sum())
+        Kc, Vc, seq_ref, stat_ref, _ = oracle.compress_append(Kc, Vc, seq_ref, stat_ref, L, k)
+    torch.cuda.synchronize()
+    assert plan.read_status(ws)[0] == 0 and triggers >= 5
+    np.testing.assert_array_equal(seq.cpu().numpy(), seq_ref)
+    np.testing.assert_array_equal(stat.cpu().numpy(), stat_ref)
+    Kn, Vn = synth.to_bits(K), synth.to_bits(V)
+    for b in range(B):
+        n = int(seq_ref[b])
+        np.testing.assert_array_equal(Kn[b, :, :n], Kc[b, :, :n])
+        np.testing.assert_array_equal(Vn[b, :, :n], Vc[b, :, :n])
+
+
 @pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("L,k,chunks", [(64, 16, 4), (256, 32, 3), (512, 128, 1)])
 def test_append_variants(binding, oracle, variant, L, k, chunks):
