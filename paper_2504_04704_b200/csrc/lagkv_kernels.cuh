@@ -264,7 +264,7 @@ __host__ __device__ constexpr size_t smem_ring_bytes(int stages) {
 template <class G>
 __host__ __device__ inline size_t smem_total_bytes(int stages, int L) {
     size_t s = smem_ring_bytes<G>(stages);         // tile rings
-    s += size_t(G::NW) * stages * 8;               // mbarriers
+    s += size_t(G::NW) * stages * 8 + 16;          // mbarriers: the rings', and two for the append move
     s += size_t(2) * G::WT * 2 * (G::D / 2) * 4;   // per-warp min/max partials
     s += sizeof(SelScratch);
     s = (s + 15) & ~size_t(15);
@@ -871,41 +871,79 @@ __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __r
         for (int j = tid; j < k; j += NT) idx_dst[dst_row0 + j] = src_row0 + kept[j];
 }
 
-// In-place move inside one cache (append): dst row = dst_row0 + j, src row = src_of(j),
-// dst <= src for every j and both ascending.  Every batch is loaded into registers by the
-// whole CTA, then a barrier, then stored, so no row is overwritten before it is read.
-template <int NT, int VPR, class SrcOf>
-__device__ void move_rows_inplace(uint16_t* K, uint16_t* V, long long ss, int dst_row0, int nrows,
-                                  SrcOf src_of, int tid) {
-    const long long items = (long long)nrows * 2 * VPR;
-    constexpr int U = 4;
-    for (long long base = 0; base < items; base += NT * U) {
-        uint4 buf[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long long i = base + u * NT + tid;
-            if (i < items) {
-                const int vec = int(i % VPR);
-                const long long r2 = i / VPR;
-                const int j = int(r2 >> 1);
-                const uint16_t* s = (r2 & 1) ? V : K;
-                buf[u] = *(reinterpret_cast<const uint4*>(s + (long long)src_of(j) * ss) + vec);
+// In-place move inside one cache (append), by one warp through the bulk-copy engine.  Row j of
+// the moved sequence (j < total) goes to row dst_row0 + j and comes from kept_pos[j] for
+// j < n_kept (the picks, ascending) and from win_src0 + j after that (the window).  Sources
+// and destinations both ascend and src >= dst for every j, so when chunks of R rows are taken
+// in order, what a chunk overwrites lies below everything a later chunk reads: the load of
+// chunk c+1 may be in flight while chunk c is stored.  Two stages of R rows of K and R rows of
+// V in shared memory (the tile rings, idle by now), one mbarrier each.  Returns false when a
+// bounded wait ran out.
+template <class G>
+__device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, long long ss, int dst_row0, int total, int n_kept,
+                               const int32_t* kept_pos, int win_src0, uint32_t stage0, int R,
+                               uint32_t bar0, int lane) {
+    constexpr uint32_t ROWB = G::D * 2;
+    const uint32_t stage_bytes = 2u * uint32_t(R) * ROWB;
+    const bool contiguous = ss == G::D;
+    const int nchunks = (total + R - 1) / R;
+    auto load = [&](int c) {
+        const int j0 = c * R, nr = min(R, total - j0);
+        const uint32_t dK = stage0 + uint32_t(c & 1) * stage_bytes, dV = dK + uint32_t(R) * ROWB;
+        const uint32_t bar = bar0 + 8 * (c & 1);
+        if (lane == 0) {
+            fence_proxy_async();
+            mbar_arrive_expect_tx(bar, 2u * uint32_t(nr) * ROWB);
+        }
+        __syncwarp();
+        if (contiguous && j0 >= n_kept) {  // window rows: one copy per tensor
+            if (lane == 0) {
+                const long long src = (long long)(win_src0 + j0) * ss;
+                bulk_g2s(dK, K + src, uint32_t(nr) * ROWB, bar);
+                bulk_g2s(dV, V + src, uint32_t(nr) * ROWB, bar);
+            }
+        } else {
+            for (int r = lane; r < nr; r += 32) {
+                const int j = j0 + r;
+                const long long src = (long long)(j < n_kept ? kept_pos[j] : win_src0 + j) * ss;
+                bulk_g2s(dK + uint32_t(r) * ROWB, K + src, ROWB, bar);
+                bulk_g2s(dV + uint32_t(r) * ROWB, V + src, ROWB, bar);
             }
         }
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long long i = base + u * NT + tid;
-            if (i < items) {
-                const int vec = int(i % VPR);
-                const long long r2 = i / VPR;
-                const int j = int(r2 >> 1);
-                uint16_t* d = (r2 & 1) ? V : K;
-                *(reinterpret_cast<uint4*>(d + (long long)(dst_row0 + j) * ss) + vec) = buf[u];
+    };
+    auto store = [&](int c) -> bool {
+        const int j0 = c * R, nr = min(R, total - j0);
+        const uint32_t sK = stage0 + uint32_t(c & 1) * stage_bytes, sV = sK + uint32_t(R) * ROWB;
+        if (!mbar_wait_bounded(bar0 + 8 * (c & 1), uint32_t(c >> 1) & 1u)) return false;
+        if (contiguous) {
+            if (lane == 0) {
+                const long long dst = (long long)(dst_row0 + j0) * ss;
+                bulk_s2g(K + dst, sK, uint32_t(nr) * ROWB);
+                bulk_s2g(V + dst, sV, uint32_t(nr) * ROWB);
+            }
+        } else {
+            for (int r = lane; r < nr; r += 32) {
+                const long long dst = (long long)(dst_row0 + j0 + r) * ss;
+                bulk_s2g(K + dst, sK + uint32_t(r) * ROWB, ROWB);
+                bulk_s2g(V + dst, sV + uint32_t(r) * ROWB, ROWB);
             }
         }
+        bulk_commit();  // every lane closes a group (empty for the lanes that stored nothing)
+        return true;
+    };
+    bool ok = true;
+    for (int c = 0; c < nchunks && ok; ++c) {
+        if (c >= 2) {  // this stage was last read by the store of chunk c-2
+            bulk_wait_read_all();
+            __syncwarp();
+        }
+        load(c);
+        if (c >= 1) ok = store(c - 1);
     }
-    __syncthreads();
+    if (ok && nchunks > 0) ok = store(nchunks - 1);
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores performed before the lengths change
+    __syncwarp();
+    return ok;
 }
 
 // ------------------------------------------------------------------------------- kernel
@@ -919,7 +957,8 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     const int NS = P.stages;
     unsigned char* ring = sm;
     uint64_t* bars = reinterpret_cast<uint64_t*>(ring + smem_ring_bytes<G>(NS));
-    uint32_t* stats = reinterpret_cast<uint32_t*>(bars + G::NW * NS);  // [2][WT][2][D/2]
+    uint64_t* move_bars = bars + G::NW * NS;  // two more for the in-place move of the append pass
+    uint32_t* stats = reinterpret_cast<uint32_t*>(move_bars + 2);  // [2][WT][2][D/2]
     SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * G::WT * 2 * (G::D / 2));
     float* sg = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
     const int Lp = (P.L + 3) & ~3;
@@ -989,7 +1028,11 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     const uint32_t bar_w = smem_u32(bars) + uint32_t(warp) * NS * 8;
     if (lane == 0)
         for (int i = 0; i < NS; ++i) mbar_init(bar_w + 8 * i, 1);
-    if (tid == 0) sc.abort = 0;
+    if (tid == 0) {
+        sc.abort = 0;
+        mbar_init(smem_u32(move_bars), 1);
+        mbar_init(smem_u32(move_bars) + 8, 1);
+    }
     fence_mbar_init();
     fence_proxy_async();
     __syncthreads();
@@ -1160,12 +1203,13 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         uint16_t* cv = const_cast<uint16_t*>(unit_base(P.V, u));
         const int n_c = n - 1;
         const int32_t* kp = P.kept_pos + (long long)u * P.max_chunks * k;
-        if (k < L) {
-            move_rows_inplace<G::NT, G::VPR>(ck, cv, P.ss, stat_rows, n_c * k,
-                                             [&](int j) { return kp[j]; }, tid);
-            const int src0 = stat_rows + n_c * L;
-            move_rows_inplace<G::NT, G::VPR>(ck, cv, P.ss, stat_rows + n_c * k, L + rem,
-                                             [&](int j) { return src0 + j; }, tid);
+        if (k < L && warp == 0) {  // kept rows, then the window, as one ascending sequence of rows
+            const int R = int(smem_ring_bytes<G>(NS) / (4 * G::D * 2));
+            if (!move_rows_bulk<G>(ck, cv, P.ss, stat_rows, n_c * k + L + rem, n_c * k, kp,
+                                   stat_rows + n_c * L - n_c * k, smem_u32(ring), R, smem_u32(move_bars), lane)) {
+                timed_out = true;
+                if (lane == 0) record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+            }
         }
         // The lengths of a sequence change once all of its heads are done: every head's CTA has
         // read the old values by then.  The last one to finish writes the new ones and clears
