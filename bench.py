@@ -35,6 +35,7 @@ DEFAULT_WORKLOAD = "llama8b_128k"
 # capture summarised under profiles/ (captured on a smaller case of the same kernel and
 # scaled by processed units where noted there); None until captured.
 NCU_TRAFFIC_BYTES = {"llama8b_128k": 21.7e9}
+NCU_TRAFFIC_BYTES_APPEND = {"decode_append": 2.234e9}    # full-size launch captured directly (one-pass metrics)
 
 
 def algorithmic_bytes(w, L_R: int, variant: int = 0) -> int:
@@ -244,8 +245,8 @@ def run_append(args, w, binding, synth, dev, local):
                    "H_kv": H, "D": D, "stored_rows": seq_trig, "static_rows": stat0, "sink": sink, "lag": L, "keep_k": k,
                    "l2": "%.2f GB touched per call, far larger than the 126 MB L2; no flush" % (alg / 1e9)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg,
-                     "kernel": "lagkv_stream_kernel"},
+                     "traffic": None if (args.layers or args.tune) else NCU_TRAFFIC_BYTES_APPEND.get(w.name),
+                     "peak_source": peak_src, "algorithmic_bytes_per_launch": alg, "kernel": "lagkv_stream_kernel"},
         "skip_call_ms": ms_skip, "clocks": clocks, "gpu_launches": args.steps,
     }))
 
