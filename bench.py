@@ -405,7 +405,8 @@ def main():
     peak, peak_src = measured_peak()
     alg = algorithmic_bytes(w, L_R, variant)
     achieved = alg / (ms_step * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES.get(w.name) if not args.layers else None
+    captured = not args.layers and not args.tune and variant == 0 and args.storage == "bf16"
+    traffic = NCU_TRAFFIC_BYTES.get(w.name) if captured else None   # counters of exactly this launch, else null
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
