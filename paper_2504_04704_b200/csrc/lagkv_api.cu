@@ -25,7 +25,11 @@ struct KernelTable {
         const KernelEntry* t;
         int c = uniform_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = uniform_dims_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = ws_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = ws_dims_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = pair_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;

@@ -22,9 +22,37 @@ struct KernelEntry {
     smem_fn_t smem;
 };
 
-// each returns the number of entries and sets *table
-int uniform_kernels(const KernelEntry** table);  // lagkv_stream_kernel: prefill and append
-int ws_kernels(const KernelEntry** table);       // lagkv_ws_kernel: warp-specialised prefill
-int pair_kernels(const KernelEntry** table);     // lagkv_pair_kernel: prefill, short partitions
+// each returns the number of entries and sets *table; the "_dims" tables hold the head
+// dimensions other than 128 (separate translation units, so that they compile side by side)
+int uniform_kernels(const KernelEntry** table);       // lagkv_stream_kernel: prefill and append
+int uniform_dims_kernels(const KernelEntry** table);
+int ws_kernels(const KernelEntry** table);            // lagkv_ws_kernel: warp-specialised prefill
+int ws_dims_kernels(const KernelEntry** table);
+int pair_kernels(const KernelEntry** table);          // lagkv_pair_kernel: prefill, short partitions
+
+// ---- table entries: (head_dim, vectors per lane, warps, tile rows, variant, element format)
+#define LAGKV_ENTRY2(D, V, NW, TR, VAR, DT) \
+    { D, NW, TR, VAR, DT, false, NW * 32, &lagkv_stream_kernel<Geo<D, V, NW, TR, DT>, VAR>, \
+      &smem_total_bytes<Geo<D, V, NW, TR, DT>> }
+#define LAGKV_ENTRY1(D, V, NW, TR, VAR) LAGKV_ENTRY2(D, V, NW, TR, VAR, 0)
+#define LAGKV_ENTRY(D, V, NW, TR) LAGKV_ENTRY1(D, V, NW, TR, 0)
+/* every uniform shape for LagKV */
+#define LAGKV_SHAPE_ENTRIES(D, V) \
+    LAGKV_ENTRY(D, V, 8, 32), LAGKV_ENTRY(D, V, 4, 32), LAGKV_ENTRY(D, V, 2, 32), LAGKV_ENTRY(D, V, 8, 16), \
+    LAGKV_ENTRY(D, V, 4, 16), LAGKV_ENTRY(D, V, 2, 16)
+/* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
+#define LAGKV_VARIANT_ENTRIES(D, V) \
+    LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
+/* fp16 caches: the planner's default shapes, every variant */
+#define LAGKV_FP16_ENTRIES(D, V) \
+    LAGKV_ENTRY2(D, V, 8, 32, 0, 1), LAGKV_ENTRY2(D, V, 4, 32, 0, 1), LAGKV_ENTRY2(D, V, 2, 16, 0, 1), \
+    LAGKV_ENTRY2(D, V, 4, 32, 1, 1), LAGKV_ENTRY2(D, V, 4, 32, 2, 1), LAGKV_ENTRY2(D, V, 2, 16, 1, 1), \
+    LAGKV_ENTRY2(D, V, 2, 16, 2, 1)
+#define LAGKV_WS_ENTRY2(D, V, NWS, TR, VAR, DT) \
+    { D, NWS + kWsEpiWarps, TR, VAR, DT, true, (NWS + kWsEpiWarps) * 32, \
+      &lagkv_ws_kernel<Geo<D, V, NWS, TR, DT>, VAR>, &ws_smem_total_bytes<Geo<D, V, NWS, TR, DT>> }
+#define LAGKV_WS_ENTRY_DT(D, V, NWS, TR, DT) \
+    LAGKV_WS_ENTRY2(D, V, NWS, TR, 0, DT), LAGKV_WS_ENTRY2(D, V, NWS, TR, 1, DT), LAGKV_WS_ENTRY2(D, V, NWS, TR, 2, DT)
+#define LAGKV_WS_ENTRY(D, V, NWS, TR) LAGKV_WS_ENTRY_DT(D, V, NWS, TR, 0)
 
 }  // namespace lagkv
