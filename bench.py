@@ -183,11 +183,9 @@ def run_append(args, w, binding, synth, dev, local):
         t = [int(x) for x in args.tune.split(",")]
         plan.tune(warps=t[0], tile_rows=t[1], stages=t[2], ctas_per_sm=t[3])
     k = plan.k
-    stat0 = sink + ((w.S - sink - L) // k) * k          # sink + whole groups of k kept rows
-    rem = 112 % L
-    if w.S - stat0 < L:
-        stat0 -= k
-    seq_trig = stat0 + 2 * L + rem                        # lengths at which every sequence triggers
+    stat0 = sink + ((w.S - sink - L) // k) * k          # the workload's stored rows: sink + groups of k kept rows
+    rem = w.S - stat0 - L                                 # + a window of L + rem rows (rem < k <= L)
+    seq_trig = stat0 + 2 * L + rem                        # L - rem new rows later every sequence triggers
     S_cap = seq_trig + 8
     K = torch.empty((Bf, H, S_cap, D), dtype=torch.bfloat16, device=dev)
     V = torch.empty_like(K)
