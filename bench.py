@@ -35,7 +35,7 @@ DEFAULT_WORKLOAD = "llama8b_128k"
 # capture summarised under profiles/ (captured on a smaller case of the same kernel and
 # scaled by processed units where noted there); None until captured.
 NCU_TRAFFIC_BYTES = {"llama8b_128k": 21.7e9}
-NCU_TRAFFIC_BYTES_APPEND = {"decode_append": 2.234e9}    # full-size launch captured directly (one-pass metrics)
+NCU_TRAFFIC_BYTES_APPEND = {"decode_append": 2.022e9}    # full-size launch captured directly (one-pass metrics)
 
 
 def algorithmic_bytes(w, L_R: int, variant: int = 0) -> int:
@@ -184,8 +184,10 @@ def run_append(args, w, binding, synth, dev, local):
         plan.tune(warps=t[0], tile_rows=t[1], stages=t[2], ctas_per_sm=t[3])
     k = plan.k
     stat0 = sink + ((w.S - sink - L) // k) * k          # the workload's stored rows: sink + groups of k kept rows
-    rem = w.S - stat0 - L                                 # + a window of L + rem rows (rem < k <= L)
-    seq_trig = stat0 + 2 * L + rem                        # L - rem new rows later every sequence triggers
+    # ... + a window of L + (w.S - stat0 - L) rows; once the new rows fill the second partition
+    # (rest = 2L, remainder 0) every sequence triggers
+    rem = 0
+    seq_trig = stat0 + 2 * L
     S_cap = seq_trig + 8
     K = torch.empty((Bf, H, S_cap, D), dtype=torch.bfloat16, device=dev)
     V = torch.empty_like(K)
