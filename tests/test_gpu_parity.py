@@ -567,6 +567,48 @@ def test_ragged_batch_prefill_in_place(binding, oracle):
         np.testing.assert_array_equal(Kn[b, :, seq[b]:], Kb[b, :, seq[b]:])
 
 
+@pytest.mark.parametrize("layout", ["padded", "bshd"])
+@pytest.mark.parametrize("L,k,chunks", [(96, 24, 2), (512, 128, 1)])
+def test_append_strided_caches(binding, oracle, layout, L, k, chunks):
+    """In-place append on caches whose rows are not contiguous: rows padded to D + 8 elements,
+    and a [B, S, H, D] cache; the bytes outside the rows (the padding) stay untouched."""
+    B, H, D, sink = 2, 3, 128, 8
+    stat = [sink, sink + 2 * k]
+    seq = [stat[0] + (chunks + 1) * L + 3, stat[1] + (chunks + 1) * L]
+    S_cap = max(seq) + 9
+    K, V = synth.make_kv(B, H, S_cap, D, seed=L + len(layout), device="cuda:0")
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    if layout == "padded":
+        Ks = torch.full((B, H, S_cap, D + 8), 7.0, dtype=torch.bfloat16, device="cuda:0")
+        Vs = torch.full_like(Ks, 7.0)
+        Ks[..., :D], Vs[..., :D] = K, V
+        strides = (H * S_cap * (D + 8), S_cap * (D + 8), D + 8)
+        view = lambda t: t[..., :D]
+    else:
+        Ks, Vs = K.permute(0, 2, 1, 3).contiguous(), V.permute(0, 2, 1, 3).contiguous()     # [B, S, H, D]
+        strides = (S_cap * H * D, D, H * D)
+        view = lambda t: t.permute(0, 2, 1, 3)
+    seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
+    stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, strides=strides, device=0)
+    ws = plan.new_workspace(chunks)
+    rc = plan.lib.lagkv_compress_append(plan.handle, binding._ptr(Ks), binding._ptr(Vs), S_cap, binding._ptr(seq_d),
+                                        binding._ptr(stat_d), chunks, None, None, binding._ptr(ws), ws.numel(),
+                                        binding._stream(torch.device("cuda", 0)))
+    assert rc == 0 and plan.read_status(ws)[0] == 0
+    Kr, Vr, seq_r, stat_r, _ = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k)
+    np.testing.assert_array_equal(seq_d.cpu().numpy(), seq_r)
+    np.testing.assert_array_equal(stat_d.cpu().numpy(), stat_r)
+    Kn, Vn = synth.to_bits(view(Ks).contiguous()), synth.to_bits(view(Vs).contiguous())
+    for b in range(B):
+        n = int(seq_r[b])
+        np.testing.assert_array_equal(Kn[b, :, :n], Kr[b, :, :n])
+        np.testing.assert_array_equal(Vn[b, :, :n], Vr[b, :, :n])
+        np.testing.assert_array_equal(Kn[b, :, seq[b]:], Kb[b, :, seq[b]:])      # beyond the old length: untouched
+    if layout == "padded":
+        assert bool((Ks[..., D:] == 7.0).all()) and bool((Vs[..., D:] == 7.0).all())
+
+
 def test_append_replays_from_a_cuda_graph(binding, oracle):
     """Decode loop: one captured launch, replayed after every appended token.  Which sequences
     compress is decided on the device from the lengths, so the graph never changes; the caches
