@@ -142,6 +142,30 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void *K, const void *V, int6
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * lagkv_compress_prefill() for caches that live in HOST memory (the same pass, Section 2.2,
+ * Eq. 7-12; the paper has no counterpart for the transfer).  K_host, V_host [B, H, S_in, D]
+ * and the outputs K_out_host, V_out_host [B, H, L_R, D], idx_out_host [B, H, L_R] are HOST
+ * pointers, contiguous, pinned if the copies are to overlap (pageable memory works, slower);
+ * the plan's strides must be 0.  The B sequences are cut into chunks of chunk_B (B % chunk_B
+ * == 0); each chunk is copied to the device, compressed and copied back, on three internal
+ * streams with two staging slots so that copies in both directions overlap the kernel.
+ *   staging    caller-owned DEVICE memory, 256-byte aligned, at least
+ *              lagkv_host_staging_bytes(plan, S_in, chunk_B) bytes (0 = bad arguments)
+ *   workspace  as for lagkv_compress_prefill()
+ * Nothing is allocated on the device; streams and events are created once per plan on the
+ * first call and freed by lagkv_plan_destroy().  Ordered after the work already on
+ * cuda_stream; cuda_stream waits for the last copy, so a synchronise on it (or
+ * lagkv_read_status) makes the host buffers valid.  The host does not block.  Calls on one
+ * plan are enqueued one at a time (internal lock) and must use the same cuda_stream if they
+ * share staging memory.
+ */
+size_t lagkv_host_staging_bytes(lagkv_plan_t plan, int64_t S_in, int32_t chunk_B);
+int lagkv_compress_prefill_host(lagkv_plan_t plan, const void *K_host, const void *V_host, int64_t S_in,
+                                void *K_out_host, void *V_out_host, int32_t *idx_out_host,
+                                int32_t chunk_B, void *staging, size_t staging_bytes, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Incremental (recursive) compression during decode or chunked prefill (Section 2.2,
  * bullets 2-4; Fig. 1).  In place on caches [B, H, S_cap, D] (the plan's strides, 0 =
  * contiguous for S_cap).  seq_len[B] and static_len[B] are DEVICE int32 arrays: rows

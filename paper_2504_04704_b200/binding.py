@@ -28,7 +28,8 @@ VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
 EXPORTS = (
     "lagkv_plan", "lagkv_plan_destroy", "lagkv_keep_count", "lagkv_compressed_len",
     "lagkv_keep_for_target", "lagkv_workspace_bytes", "lagkv_workspace_init",
-    "lagkv_compress_prefill", "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
+    "lagkv_compress_prefill", "lagkv_compress_prefill_host", "lagkv_host_staging_bytes",
+    "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
     "lagkv_read_status",
     "lagkv_launch_info", "lagkv_plan_tune", "lagkv_selftest_bounded_wait", "lagkv_status_string", "lagkv_version",
 )
@@ -81,6 +82,10 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_workspace_init.argtypes = [vp, vp, sz, vp]
     lib.lagkv_compress_prefill.restype = ctypes.c_int
     lib.lagkv_compress_prefill.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+    lib.lagkv_host_staging_bytes.restype = sz
+    lib.lagkv_host_staging_bytes.argtypes = [vp, i64, i32]
+    lib.lagkv_compress_prefill_host.restype = ctypes.c_int
+    lib.lagkv_compress_prefill_host.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, vp, sz, vp, sz, vp]
     lib.lagkv_compress_append.restype = ctypes.c_int
     lib.lagkv_compress_append.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.lagkv_compress_append_noalloc.restype = ctypes.c_int
@@ -347,63 +352,46 @@ class ChunkedPrefill:
 
 
 class HostPrefill:
-    """Prefill compression of a cache that lives in pinned HOST memory.
+    """Prefill compression of a cache that lives in pinned HOST memory: ``lagkv_compress_prefill_host``.
 
-    The ``[B, H, S_in, D]`` host cache is cut into chunks of ``chunk_B`` sequences (or
-    layers folded into B).  Each chunk is copied to a device staging buffer, compressed with
-    ``lagkv_compress_prefill`` and its compacted rows and indices are copied back; the three
-    stages run on three streams with two staging slots so that copies in both directions
-    overlap the kernel.  All arithmetic is the CUDA library's.
+    The library cuts the ``[B, H, S_in, D]`` host cache into chunks of ``chunk_B`` sequences (or
+    layers folded into B), copies each chunk to the device staging buffer held here, compresses
+    it and copies the compacted rows and indices back, on three streams with two staging slots
+    so that copies in both directions overlap the kernel.  This class only owns the staging
+    buffer and the workspace and marshals the call.
     """
 
     def __init__(self, B, H_kv, D, S_in, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1, chunk_B=1, device=0):
         if B % chunk_B:
             raise ValueError("B must be a multiple of chunk_B")
         self.B, self.chunk_B, self.S_in = int(B), int(chunk_B), int(S_in)
-        self.plan = Plan(chunk_B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof,
-                         device=device)
+        self.plan = Plan(B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof, device=device)
         dev = self.plan._dev()
         self.L_R = self.plan.compressed_len(S_in)
         self.ws = self.plan.new_workspace()
-        mk = lambda *shape, dt=torch.bfloat16: torch.empty(shape, dtype=dt, device=dev)
-        self.slots = [dict(K=mk(chunk_B, H_kv, S_in, D), V=mk(chunk_B, H_kv, S_in, D),
-                           K_out=mk(chunk_B, H_kv, self.L_R, D), V_out=mk(chunk_B, H_kv, self.L_R, D),
-                           idx=mk(chunk_B, H_kv, self.L_R, dt=torch.int32)) for _ in range(2)]
-        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream(dev) for _ in range(3))
+        nbytes = int(self.plan.lib.lagkv_host_staging_bytes(self.plan.handle, self.S_in, self.chunk_B))
+        if nbytes == 0:
+            raise LagKVError(LAGKV_EINVAL, "lagkv_host_staging_bytes")
+        self.staging = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         self.h2d_bytes = 2 * B * H_kv * S_in * D * 2
         self.d2h_bytes = 2 * B * H_kv * self.L_R * D * 2 + B * H_kv * self.L_R * 4
 
-    def run(self, K_host, V_host, K_out_host, V_out_host, idx_host) -> None:
-        """All five tensors are pinned host tensors; returns after the last copy has landed."""
-        cb = self.chunk_B
-        comp_done = [None, None]
-        out_done = [None, None]
-        cur = torch.cuda.current_stream(self.plan._dev())
-        for s in (self.s_in, self.s_comp, self.s_out):
-            s.wait_stream(cur)
-        for c in range(self.B // cb):
-            slot = self.slots[c % 2]
-            sl = slice(c * cb, (c + 1) * cb)
-            with torch.cuda.stream(self.s_in):
-                if comp_done[c % 2] is not None:
-                    self.s_in.wait_event(comp_done[c % 2])
-                slot["K"].copy_(K_host[sl], non_blocking=True)
-                slot["V"].copy_(V_host[sl], non_blocking=True)
-                in_done = torch.cuda.Event()
-                in_done.record(self.s_in)
-            with torch.cuda.stream(self.s_comp):
-                self.s_comp.wait_event(in_done)
-                if out_done[c % 2] is not None:
-                    self.s_comp.wait_event(out_done[c % 2])
-                self.plan.compress_prefill(slot["K"], slot["V"], self.ws, out=slot, want_scores=False)
-                comp_done[c % 2] = torch.cuda.Event()
-                comp_done[c % 2].record(self.s_comp)
-            with torch.cuda.stream(self.s_out):
-                self.s_out.wait_event(comp_done[c % 2])
-                K_out_host[sl].copy_(slot["K_out"], non_blocking=True)
-                V_out_host[sl].copy_(slot["V_out"], non_blocking=True)
-                idx_host[sl].copy_(slot["idx"], non_blocking=True)
-                out_done[c % 2] = torch.cuda.Event()
-                out_done[c % 2].record(self.s_out)
-        cur.wait_stream(self.s_out)
-        self.s_out.synchronize()
+    def run(self, K_host, V_host, K_out_host, V_out_host, idx_host, wait: bool = True) -> None:
+        """All five tensors are contiguous (pinned) host tensors.  The call only enqueues; with
+        ``wait`` it returns after the last copy has landed."""
+        want = {"K_host": (K_host, (self.B, self.plan.cfg.H_kv, self.S_in, self.plan.cfg.D), torch.bfloat16),
+                "V_host": (V_host, (self.B, self.plan.cfg.H_kv, self.S_in, self.plan.cfg.D), torch.bfloat16),
+                "K_out_host": (K_out_host, (self.B, self.plan.cfg.H_kv, self.L_R, self.plan.cfg.D), torch.bfloat16),
+                "V_out_host": (V_out_host, (self.B, self.plan.cfg.H_kv, self.L_R, self.plan.cfg.D), torch.bfloat16),
+                "idx_host": (idx_host, (self.B, self.plan.cfg.H_kv, self.L_R), torch.int32)}
+        for name, (t, shape, dt) in want.items():
+            if t.is_cuda or t.dtype != dt or tuple(t.shape) != shape or not t.is_contiguous():
+                raise TypeError(f"{name} must be a contiguous host tensor {shape} of {dt}")
+        dev = self.plan._dev()
+        rc = self.plan.lib.lagkv_compress_prefill_host(
+            self.plan.handle, _ptr(K_host), _ptr(V_host), self.S_in, _ptr(K_out_host), _ptr(V_out_host),
+            _ptr(idx_host), self.chunk_B, _ptr(self.staging), self.staging.numel(), _ptr(self.ws), self.ws.numel(),
+            _stream(dev))
+        _check(rc, "lagkv_compress_prefill_host")
+        if wait:
+            torch.cuda.current_stream(dev).synchronize()

@@ -73,6 +73,27 @@ struct lagkv_plan_s {
     Shape pair;       // pair kernel, preferred for short partitions with enough of them (kidx < 0: none)
     bool tuned;       // lagkv_plan_tune() fixed the prefill kernel: no switching by size
     Shape app;        // kernel used by lagkv_compress_append (always the uniform kernel)
+    // lagkv_compress_prefill_host(): three streams and the events between them, made on first use
+    std::mutex host_mu;
+    bool host_ready = false;
+    cudaStream_t host_stream[3] = {nullptr, nullptr, nullptr};  // copy in, compute, copy out
+    cudaEvent_t host_start = nullptr, host_in[2] = {nullptr, nullptr}, host_comp[2] = {nullptr, nullptr},
+                host_out[2] = {nullptr, nullptr};
+    ~lagkv_plan_s() {
+        if (!host_stream[0] && !host_start) return;
+        int prev = -1;
+        const bool sw = cfg.device >= 0 && cudaGetDevice(&prev) == cudaSuccess && prev != cfg.device &&
+                        cudaSetDevice(cfg.device) == cudaSuccess;
+        for (int i = 0; i < 3; ++i)
+            if (host_stream[i]) cudaStreamDestroy(host_stream[i]);
+        if (host_start) cudaEventDestroy(host_start);
+        for (int i = 0; i < 2; ++i) {
+            if (host_in[i]) cudaEventDestroy(host_in[i]);
+            if (host_comp[i]) cudaEventDestroy(host_comp[i]);
+            if (host_out[i]) cudaEventDestroy(host_out[i]);
+        }
+        if (sw) cudaSetDevice(prev);
+    }
 };
 
 namespace {
@@ -286,9 +307,10 @@ int lagkv_workspace_init(lagkv_plan_t plan, void* workspace, size_t workspace_by
     return LAGKV_OK;
 }
 
-int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, void* K_out,
-                           void* V_out, int32_t* idx_out, float* scores_out, void* workspace,
-                           size_t workspace_bytes, void* cuda_stream) {
+// lagkv_compress_prefill() for the first B sequences of the plan (the host pipeline runs it chunk by chunk)
+static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, int64_t S_in, void* K_out,
+                        void* V_out, int32_t* idx_out, float* scores_out, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
     if (plan == nullptr || K == nullptr || V == nullptr || plan->cfg.device < 0) return LAGKV_EINVAL;
     if ((K_out == nullptr) != (V_out == nullptr)) return LAGKV_EINVAL;
     if (S_in < 0 || S_in > 0x7fffffffll - 65536) return LAGKV_EINVAL;
@@ -305,7 +327,7 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
 
     DeviceGuard guard(c.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const long long U = (long long)c.B * c.H_kv;
+    const long long U = (long long)B * c.H_kv;
     const int64_t rest = S_in - c.sink;
 
     if (rest < 2ll * c.lag) {  // pass skipped: identity
@@ -332,7 +354,7 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
     P.sb = st.sb;
     P.sh = st.sh;
     P.ss = st.ss;
-    P.B = c.B;
+    P.B = B;
     P.H = c.H_kv;
     P.L = c.lag;
     P.k = plan->k;
@@ -357,6 +379,118 @@ int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int6
                          shape.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
     return check_launch();
+}
+
+int lagkv_compress_prefill(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, void* K_out,
+                           void* V_out, int32_t* idx_out, float* scores_out, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    if (plan == nullptr) return LAGKV_EINVAL;
+    return prefill_impl(plan, plan->cfg.B, K, V, S_in, K_out, V_out, idx_out, scores_out, workspace, workspace_bytes,
+                        cuda_stream);
+}
+
+// ---- host-resident caches ------------------------------------------------------------------
+namespace {
+size_t round256(size_t v) { return (v + 255) & ~size_t(255); }
+struct HostSlot {  // byte offsets of one staging slot
+    size_t K, V, K_out, V_out, idx, total;
+};
+HostSlot host_slot_layout(const lagkv_plan_s* plan, int64_t S_in, int chunk_B, int64_t L_R) {
+    const size_t units = size_t(chunk_B) * plan->cfg.H_kv, row = size_t(plan->cfg.D) * 2;
+    HostSlot h;
+    h.K = 0;
+    h.V = h.K + round256(units * S_in * row);
+    h.K_out = h.V + round256(units * S_in * row);
+    h.V_out = h.K_out + round256(units * L_R * row);
+    h.idx = h.V_out + round256(units * L_R * row);
+    h.total = h.idx + round256(units * L_R * sizeof(int32_t));
+    return h;
+}
+int host_pipe_make(lagkv_plan_s* plan) {  // caller holds host_mu and has set the device
+    if (plan->host_ready) return LAGKV_OK;
+    bool ok = true;
+    for (int i = 0; i < 3; ++i)
+        ok = ok && cudaStreamCreateWithFlags(&plan->host_stream[i], cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&plan->host_start, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2; ++i) {
+        ok = ok && cudaEventCreateWithFlags(&plan->host_in[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&plan->host_comp[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&plan->host_out[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    plan->host_ready = ok;
+    return ok ? LAGKV_OK : LAGKV_ECUDA;
+}
+}  // namespace
+
+size_t lagkv_host_staging_bytes(lagkv_plan_t plan, int64_t S_in, int32_t chunk_B) {
+    if (plan == nullptr || S_in < 1 || S_in > 0x7fffffffll - 65536 || chunk_B < 1 || chunk_B > plan->cfg.B) return 0;
+    return 2 * host_slot_layout(plan, S_in, chunk_B, lagkv_compressed_len(plan, S_in, -1)).total;
+}
+
+int lagkv_compress_prefill_host(lagkv_plan_t plan, const void* K_host, const void* V_host, int64_t S_in,
+                                void* K_out_host, void* V_out_host, int32_t* idx_out_host, int32_t chunk_B,
+                                void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream) {
+    if (plan == nullptr || K_host == nullptr || V_host == nullptr || K_out_host == nullptr || V_out_host == nullptr ||
+        idx_out_host == nullptr || plan->cfg.device < 0)
+        return LAGKV_EINVAL;
+    const lagkv_config& c = plan->cfg;
+    if (S_in < 1 || S_in > 0x7fffffffll - 65536 || chunk_B < 1 || (c.B % chunk_B) != 0) return LAGKV_EINVAL;
+    if (c.stride_b != 0 || c.stride_h != 0 || c.stride_s != 0) return LAGKV_EINVAL;  // host caches are contiguous
+    if (staging == nullptr || (reinterpret_cast<uintptr_t>(staging) & 255u)) return LAGKV_EINVAL;
+    if (workspace == nullptr || workspace_bytes < kStatusWords * sizeof(int32_t)) return LAGKV_EWORKSPACE;
+    const int64_t L_R = lagkv_compressed_len(plan, S_in, -1);
+    const HostSlot lay = host_slot_layout(plan, S_in, chunk_B, L_R);
+    if (staging_bytes < 2 * lay.total) return LAGKV_EWORKSPACE;
+
+    DeviceGuard guard(c.device);
+    std::lock_guard<std::mutex> lock(plan->host_mu);  // one pipeline per plan: calls enqueue one after another
+    if (host_pipe_make(plan) != LAGKV_OK) return LAGKV_ECUDA;
+    cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+    cudaStream_t s_in = plan->host_stream[0], s_comp = plan->host_stream[1], s_out = plan->host_stream[2];
+    bool ok = cudaEventRecord(plan->host_start, user) == cudaSuccess;
+    for (int i = 0; i < 3; ++i) ok = ok && cudaStreamWaitEvent(plan->host_stream[i], plan->host_start, 0) == cudaSuccess;
+
+    const size_t units = size_t(chunk_B) * c.H_kv, row = size_t(c.D) * 2;
+    const size_t in_bytes = units * S_in * row, out_bytes = units * L_R * row, idx_bytes = units * L_R * sizeof(int32_t);
+    const int chunks = c.B / chunk_B;
+    int rc = LAGKV_OK;
+    for (int ch = 0; ch < chunks && ok && rc == LAGKV_OK; ++ch) {
+        const int sl = ch & 1;
+        unsigned char* base = static_cast<unsigned char*>(staging) + size_t(sl) * lay.total;
+        const unsigned char* kh = static_cast<const unsigned char*>(K_host) + size_t(ch) * in_bytes;
+        const unsigned char* vh = static_cast<const unsigned char*>(V_host) + size_t(ch) * in_bytes;
+        // copy in: the slot's inputs are free once the kernel of chunk ch-2 is done
+        if (ch >= 2) ok = ok && cudaStreamWaitEvent(s_in, plan->host_comp[sl], 0) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(base + lay.K, kh, in_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(base + lay.V, vh, in_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        ok = ok && cudaEventRecord(plan->host_in[sl], s_in) == cudaSuccess;
+        // compute: the slot's outputs are free once chunk ch-2 has been copied out
+        ok = ok && cudaStreamWaitEvent(s_comp, plan->host_in[sl], 0) == cudaSuccess;
+        if (ch >= 2) ok = ok && cudaStreamWaitEvent(s_comp, plan->host_out[sl], 0) == cudaSuccess;
+        if (ok)
+            rc = prefill_impl(plan, chunk_B, base + lay.K, base + lay.V, S_in, base + lay.K_out, base + lay.V_out,
+                              reinterpret_cast<int32_t*>(base + lay.idx), nullptr, workspace, workspace_bytes, s_comp);
+        ok = ok && cudaEventRecord(plan->host_comp[sl], s_comp) == cudaSuccess;
+        // copy out
+        ok = ok && cudaStreamWaitEvent(s_out, plan->host_comp[sl], 0) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(static_cast<unsigned char*>(K_out_host) + size_t(ch) * out_bytes, base + lay.K_out,
+                                   out_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(static_cast<unsigned char*>(V_out_host) + size_t(ch) * out_bytes, base + lay.V_out,
+                                   out_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(reinterpret_cast<unsigned char*>(idx_out_host) + size_t(ch) * idx_bytes,
+                                   base + lay.idx, idx_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        ok = ok && cudaEventRecord(plan->host_out[sl], s_out) == cudaSuccess;
+    }
+    // the caller's stream continues when everything enqueued above is done (also after an error,
+    // so that the staging buffers are never reused under a copy still in flight)
+    for (int sl = 0; sl < 2 && sl < chunks; ++sl) {
+        cudaStreamWaitEvent(user, plan->host_out[sl], 0);
+        cudaStreamWaitEvent(user, plan->host_comp[sl], 0);
+        cudaStreamWaitEvent(user, plan->host_in[sl], 0);
+    }
+    if (rc != LAGKV_OK) return rc;
+    return ok ? LAGKV_OK : LAGKV_ECUDA;
 }
 
 int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,

@@ -887,6 +887,25 @@ def test_host_prefill_pipeline_matches_direct_call(binding, oracle):
     ref = oracle.compress(synth.to_bits(K), synth.to_bits(V), sink, L, k)
     np.testing.assert_array_equal(Io.numpy(), ref["idx"])
     np.testing.assert_array_equal(synth.to_bits(Ko), ref["K_out"])
+    assert hp.plan.read_status(hp.ws)[0] == 0
+    # one chunk only, and a cache too short to compress (identity), through the same entry point
+    for chunk_B, S2 in ((B, S), (3, sink + 2 * L - 1)):
+        hp2 = binding.HostPrefill(B, H, D, S2, sink, L, keep_k=k, chunk_B=chunk_B, device=0)
+        Kh2, Vh2 = Kh[:, :, :S2].contiguous().pin_memory(), Vh[:, :, :S2].contiguous().pin_memory()
+        Ko2 = torch.zeros((B, H, hp2.L_R, D), dtype=torch.bfloat16).pin_memory()
+        Vo2, Io2 = torch.zeros_like(Ko2).pin_memory(), torch.zeros((B, H, hp2.L_R), dtype=torch.int32).pin_memory()
+        hp2.run(Kh2, Vh2, Ko2, Vo2, Io2)
+        ref2 = oracle.compress(synth.to_bits(Kh2), synth.to_bits(Vh2), sink, L, k)
+        np.testing.assert_array_equal(Io2.numpy(), ref2["idx"])
+        np.testing.assert_array_equal(synth.to_bits(Ko2), ref2["K_out"])
+        np.testing.assert_array_equal(synth.to_bits(Vo2), ref2["V_out"])
+    # a staging buffer that is too small is refused before anything is enqueued
+    rc = hp.plan.lib.lagkv_compress_prefill_host(
+        hp.plan.handle, binding._ptr(Kh), binding._ptr(Vh), S, binding._ptr(Ko), binding._ptr(Vo), binding._ptr(Io), 2,
+        binding._ptr(hp.staging), hp.staging.numel() - 256, binding._ptr(hp.ws), hp.ws.numel(),
+        binding._stream(torch.device("cuda", 0)))
+    assert rc == binding.LAGKV_EWORKSPACE
+    assert hp.plan.lib.lagkv_host_staging_bytes(hp.plan.handle, S, B + 1) == 0      # more than the plan holds
 
 
 def test_bounded_wait_gives_up_and_reports(binding):
