@@ -355,6 +355,16 @@ def main():
         torch.cuda.synchronize()
         ms_total = sum(a.elapsed_time(b) for a, b in evs)
     wall1 = time.time()
+    # spread of single steps (outside the timed region: an event pair around every launch)
+    per = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+    for a, b in per:
+        if flush_l2:
+            scrub.fill_(1)
+        a.record(stream)
+        step()
+        b.record(stream)
+    torch.cuda.synchronize()
+    per_ms = sorted(a.elapsed_time(b) for a, b in per)
     if world > 1:
         dist.barrier()
     status = plan.read_status(ws)
@@ -411,6 +421,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "single_steps_ms": {"median": per_ms[len(per_ms) // 2], "min": per_ms[0], "max": per_ms[-1], "n": len(per_ms),
+                            "note": "this rank, 20 launches timed one by one after the timed region"},
         "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
                    "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio, "keep_k": plan.k, "L_R": L_R,
                    "variant": args.variant,
