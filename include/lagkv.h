@@ -46,7 +46,7 @@ typedef struct lagkv_plan_s *lagkv_plan_t;
 enum lagkv_status {
     LAGKV_OK = 0,
     LAGKV_EINVAL = 1,       /* null pointer, misalignment, bad shape / stride / size  */
-    LAGKV_EUNSUPPORTED = 2, /* valid request this build has no kernel for             */
+    LAGKV_EUNSUPPORTED = 2, /* valid request the library has no kernel for            */
     LAGKV_EWORKSPACE = 3,   /* workspace missing or too small                         */
     LAGKV_ECUDA = 4,        /* CUDA runtime error at launch (left sticky, not cleared)*/
     LAGKV_ETIMEOUT = 5,     /* device: a bounded wait on an async copy ran out        */

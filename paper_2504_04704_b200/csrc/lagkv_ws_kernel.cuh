@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 bad = true;
                 raise_abort();
             }
-            dead = named_bar_or(kBarSelect, kWsSelThreads, bad);  // one verdict for the group
+            dead = named_bar_or(kBarSelect, kWsSelThreads, bad);  // one decision for the group
             if (score && !dead) {
                 float* sg0 = sgbase + (buf * 2) * Lp;
                 float* sg1 = sg0 + Lp;
