@@ -94,3 +94,16 @@ def test_launch_shapes_fit_the_sm(binding):
     assert plan.launch_info(100)["smem"] == 0        # identity pass: plain copy kernel
     with pytest.raises(binding.LagKVError):
         plan.tune(warps=8, tile_rows=32, stages=8)   # 512 KiB of ring does not fit
+
+
+def test_plain_c_program_links_and_runs(binding, tmp_path):
+    """include/lagkv.h is valid strict C99 and a C program linked to the shared object gets the
+    planner's integers (host-side calls only: no GPU needed)."""
+    import subprocess
+    lib = Path(binding.LIB_PATH)
+    exe = tmp_path / "host_only"
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", f"-I{ROOT / 'include'}",
+                    str(ROOT / "tests" / "c_abi" / "host_only.c"), "-o", str(exe), f"-L{lib.parent}",
+                    f"-l:{lib.name}", f"-Wl,-rpath,{lib.parent}"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", out.stderr
