@@ -948,3 +948,21 @@ def test_argument_errors(binding):
         plan.compress_prefill(K, V, ws, out={"K_out": K, "V_out": V})
     assert e.value.code == binding.LAGKV_EINVAL
     assert plan.read_status(ws)[0] == 0
+
+
+def test_c_program_prefill_parity(binding, tmp_path):
+    """No Python between the library and the oracle: a C program (tests/c_abi/prefill_parity.c)
+    allocates with the CUDA runtime, calls the C ABI, and compares with the C oracle linked in."""
+    import os
+    import subprocess
+    from pathlib import Path
+    root = Path(__file__).resolve().parent.parent
+    lib = Path(binding.LIB_PATH)
+    cuda = Path(os.environ.get("CUDA_HOME", "/usr/local/cuda"))
+    exe = tmp_path / "prefill_parity"
+    subprocess.run(["gcc", "-std=c99", "-O2", "-Wall", "-Werror", "-fopenmp", f"-I{root / 'include'}", f"-I{cuda / 'include'}",
+                    str(root / "tests" / "c_abi" / "prefill_parity.c"), str(root / "oracle" / "lagkv_oracle.c"),
+                    "-o", str(exe), f"-L{lib.parent}", f"-l:{lib.name}", f"-Wl,-rpath,{lib.parent}",
+                    f"-L{cuda / 'lib64'}", "-lcudart", f"-Wl,-rpath,{cuda / 'lib64'}", "-lm"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.startswith("ok"), out.stdout + out.stderr
