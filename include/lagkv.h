@@ -63,7 +63,7 @@ enum lagkv_variant {
 
 enum lagkv_dtype {
     LAGKV_DTYPE_BF16 = 0, /* the default (a zeroed field)                                */
-    LAGKV_DTYPE_FP16 = 1  /* IEEE binary16 caches; compiled for head_dim 128             */
+    LAGKV_DTYPE_FP16 = 1  /* IEEE binary16 caches                                        */
 };
 
 typedef struct {

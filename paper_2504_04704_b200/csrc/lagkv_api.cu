@@ -27,6 +27,10 @@ struct KernelTable {
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = uniform_dims_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = uniform_dims_fp16_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = ws_dims_fp16_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = ws_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = ws_dims_kernels(&t);

@@ -11,6 +11,7 @@ namespace {
 const KernelEntry kTable[] = {
     LAGKV_PAIR_ENTRY(128, 2, 32), LAGKV_PAIR_ENTRY(128, 2, 16), LAGKV_PAIR_ENTRY(64, 1, 32), LAGKV_PAIR_ENTRY(256, 2, 16),
     LAGKV_PAIR_ENTRY(96, 3, 32), LAGKV_PAIR_ENTRY_DT(128, 2, 32, 1),
+    LAGKV_PAIR_ENTRY_DT(64, 1, 32, 1), LAGKV_PAIR_ENTRY_DT(256, 2, 16, 1), LAGKV_PAIR_ENTRY_DT(96, 3, 32, 1),
 };
 }  // namespace
 

@@ -26,8 +26,10 @@ struct KernelEntry {
 // dimensions other than 128 (separate translation units, so that they compile side by side)
 int uniform_kernels(const KernelEntry** table);       // lagkv_stream_kernel: prefill and append
 int uniform_dims_kernels(const KernelEntry** table);
+int uniform_dims_fp16_kernels(const KernelEntry** table);
 int ws_kernels(const KernelEntry** table);            // lagkv_ws_kernel: warp-specialised prefill
 int ws_dims_kernels(const KernelEntry** table);
+int ws_dims_fp16_kernels(const KernelEntry** table);
 int pair_kernels(const KernelEntry** table);          // lagkv_pair_kernel: prefill, short partitions
 
 // ---- table entries: (head_dim, vectors per lane, warps, tile rows, variant, element format)

@@ -443,10 +443,26 @@ def test_fp16_and_bf16_agree_on_values_both_hold(binding):
     assert torch.equal(res[0]["K_out"].float(), res[1]["K_out"].float())
 
 
-def test_fp16_shapes_refused(binding):
-    with pytest.raises(binding.LagKVError) as e:
-        binding.Plan(1, 2, 64, 4, 64, device=0, dtype=torch.float16)       # fp16 is compiled for head_dim 128
-    assert e.value.code == binding.LAGKV_EUNSUPPORTED
+@pytest.mark.parametrize("D", [64, 96, 256])
+@pytest.mark.parametrize("L,k,tune", [(64, 16, None), (128, 16, "pairs"), (256, 64, None)])
+def test_fp16_head_dims(binding, oracle, D, L, k, tune):
+    tune = PAIRS if tune == "pairs" else tune
+    if tune is PAIRS and D == 256:
+        tune = dict(PAIRS, tile_rows=16)
+    run_prefill(binding, oracle, 12 if tune else 2, 3, D, 4 + 7 * L + 33, 4, L, k, seed=D + L, tune=tune,
+                dtype=torch.float16)
+
+
+def test_fp16_append_head_dims(binding, oracle):
+    for D in (64, 96, 256):
+        sink, L, k = 8, 96, 24
+        stat = [sink, sink + 3 * k]
+        seq = [stat[0] + 3 * L + 3, stat[1] + 2 * L]
+        check_append(append_case(binding, oracle, 2, 3, D, seq[0] + 9, sink, L, k, seq, stat, 2, seed=D,
+                                 dtype=torch.float16), 2)
+
+
+def test_fp16_tensor_type_is_checked(binding):
     plan = binding.Plan(1, 2, 128, 4, 64, device=0, dtype=torch.float16)
     K, V = synth.make_kv(1, 2, 300, 128, seed=1, device="cuda:0")
     with pytest.raises(TypeError):
