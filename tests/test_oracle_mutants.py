@@ -30,6 +30,11 @@ MUTANTS = {
     "tie_to_higher_index": ("score[t] > score[best]) best = t;", "score[t] >= score[best]) best = t;"),
     "partition_count_rounded_up": ("int64_t n = rest / L;\n    int64_t rem", "int64_t n = (rest + L - 1) / L;\n    int64_t rem"),
     "l2_not_negated": ("score[t] = -sqrt(ss);", "score[t] = sqrt(ss);"),
+    "fp16_exponent_bias": ("ldexp(1.0 + (double)frac / 1024.0, e - 15);", "ldexp(1.0 + (double)frac / 1024.0, e - 16);"),
+    "fp16_subnormal_scale": ("ldexp((double)frac, -24);", "ldexp((double)frac, -25);"),
+    "fp16_fraction_width": ("(double)frac / 1024.0", "(double)frac / 2048.0"),
+    "storage_flag_ignored": ("return storage == LAGKV_ORACLE_FP16 ? fp16_to_double(bits) : bf16_to_double(bits);",
+                             "return bf16_to_double(bits);"),
 }
 
 
@@ -57,6 +62,9 @@ def run_pins(mod, only=None):
         ("ddof_matters", lambda: pins.test_ddof_matters(mod)),
         ("l2", lambda: pins.test_l2norm_variant(mod)),
         ("brute", lambda: pins.test_c_oracle_vs_python_brute(mod, 0, 1)),
+        ("decode", lambda: pins.test_decode_every_bit_pattern(mod)),
+        ("fp16_same_values", lambda: pins.test_fp16_storage_same_values_same_result(mod, 1)),
+        ("fp16_only", lambda: pins.test_fp16_storage_values_only_fp16_holds(mod)),
     ]
     failed = []
     for name, fn in checks:
