@@ -374,6 +374,10 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
     P.total_slots = U * P.spu;
     const Shape& shape = prefill_shape(plan, P.total_slots);
     P.stages = shape.stages;
+    // Measured on the Ls = 65536 sweep and the 32K / 128K configurations: with L >= 1024 and
+    // 1/8 <= k/L <= 1/4 the select warps gain 2-7 % by moving every second partition's kept rows;
+    // with shorter partitions (or more rows to move) they fall behind the streamers (-4 to -25 %).
+    P.sel_emit = (c.lag >= 1024 && 4 * plan->k <= c.lag && 8 * plan->k >= c.lag) ? 1 : 0;
 
     const KernelEntry& ke = kKernels[shape.kidx];
     long long grid = (long long)plan->sm_count * shape.ctas_per_sm;

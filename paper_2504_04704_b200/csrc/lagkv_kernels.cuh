@@ -50,6 +50,7 @@ struct Params {
     int spu;                      // prefill, warp-specialised kernel: slots per (b, h) unit
     int max_chunks;               // append
     int stages;                   // ring depth per warp
+    int sel_emit;                 // warp-specialised kernel: select warps move the kept rows of odd slots
 };
 
 // ------------------------------------------------------------------------------ PTX helpers

@@ -87,6 +87,10 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     auto slot_part = [&](int j) -> int { return local_stats ? n - 2 - (j >> 1) : (l2norm ? n - 2 - j : n - 1 - j); };
     auto slot_scored = [&](int j) -> bool { return local_stats ? (j & 1) != 0 : (l2norm || j != 0); };
     auto slot_needs_prev = [&](int j) -> bool { return !l2norm && slot_scored(j); };
+    // Slots (counted from the first one this CTA streams) whose kept rows the select warps move
+    // themselves: every second one where the host found that they have the time (P.sel_emit).
+    const bool sel_emit = P.sel_emit != 0;
+    auto sel_moves = [&](long long i) -> bool { return sel_emit && (i & 1) != 0; };
     const bool extra = s_first < s_hi && slot_needs_prev(int(s_first % spu));
     const long long s_lo = extra ? s_first - 1 : s_first;
 
@@ -292,16 +296,16 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     const int row0 = sink + p * L;
                     if (P.idx_out != nullptr) {
                         for (int j = etid; j < k; j += kWsSelThreads) P.idx_out[o + j] = row0 + kept[j];
-                    } else if (P.K_out != nullptr && !(i & 1)) {
+                    } else if (P.K_out != nullptr && !sel_moves(i)) {
                         for (int j = etid; j < k; j += kWsSelThreads)
                             *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::D) = row0 + kept[j];
                     }
                 }
-                // Odd slots: the select warps, idle most of the time, move the kept rows themselves
-                // while kept[] is at hand (even slots are left to the copy warp and the gather
-                // phase).  Every second slot is what they can carry without holding up the
-                // streamers; it takes a fifth of the rows off the gather phase.
-                if ((i & 1) && P.K_out != nullptr)
+                // Long partitions: the select warps, idle most of the time, move the kept rows of
+                // odd slots themselves while kept[] is at hand (the others are left to the copy
+                // warp and the gather phase).  Every second slot is what they can carry without
+                // holding up the streamers; with short partitions they have no time to spare.
+                if (sel_moves(i) && P.K_out != nullptr)
                     emit_kept<kWsSelThreads, G::VPR, 16>(unit_base(P.K, u), unit_base(P.V, u), P.ss,
                                                          P.K_out + (long long)u * P.L_R * G::D,
                                                          P.V_out + (long long)u * P.L_R * G::D, sink + p * L,
@@ -353,7 +357,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                     // and the odd slots, whose rows the select warps move
                     while (gslot < nslots) {
                         const long long sl = s_lo + gslot;
-                        if (slot_scored(int(sl % spu)) && sl >= s_first && !(gslot & 1)) break;
+                        if (slot_scored(int(sl % spu)) && sl >= s_first && !sel_moves(gslot)) break;
                         ++gslot;
                     }
                     if (gslot < done && done < nslots) {
@@ -468,7 +472,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         const long long s_from = s_lo + *reinterpret_cast<volatile int*>(&sc.claimed);
         for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
             const int u = int(s / spu), sj = int(s % spu), p = slot_part(sj);
-            if (!slot_scored(sj) || ((s - s_lo) & 1)) continue;  // odd slots: done by the select warps
+            if (!slot_scored(sj) || sel_moves(s - s_lo)) continue;  // done by the select warps
             const uint16_t* srcK = unit_base(P.K, u);
             const uint16_t* srcV = unit_base(P.V, u);
             const long long o = (long long)u * P.L_R + sink + p * k;
