@@ -161,7 +161,7 @@ int first_fit(const lagkv_plan_s* pl, const Cand* cands, int nc, Shape* out) {
 // CTA per (b, h).
 int choose_shape(lagkv_plan_s* pl) {
     const int L = pl->cfg.lag;
-    Cand uni[8];
+    Cand uni[10];
     int nu = 0;
     if (L >= 1024 && pl->cfg.variant == LAGKV_VARIANT_LAGKV) {  // eight-warp CTAs are compiled for LagKV only
         uni[nu++] = {8, 32, 3, 1};
@@ -171,6 +171,7 @@ int choose_shape(lagkv_plan_s* pl) {
         uni[nu++] = {4, 32, 3, 2};
         uni[nu++] = {4, 32, 2, 2};
     }
+    uni[nu++] = {2, 16, 2, 6};  // two stages: 3-4 % ahead of three on the short-partition sweep cells
     uni[nu++] = {2, 16, 3, 6};
     uni[nu++] = {2, 16, 3, 4};
     uni[nu++] = {2, 16, 2, 2};
@@ -191,7 +192,9 @@ int choose_shape(lagkv_plan_s* pl) {
     // time (measured on the Ls = 65536 sweep).  Whether there are enough partitions to feed
     // them is known only at the call.
     if (pl->cfg.variant == LAGKV_VARIANT_LAGKV && ((L <= 128 && 4 * pl->k <= L) || (L <= 256 && 8 * pl->k <= L))) {
-        const Cand pr[] = {{LAGKV_TUNE_PAIRS, 32, 2, 1}, {LAGKV_TUNE_PAIRS, 16, 2, 1}};
+        // 16-row tiles when many rows are kept (2-5 % on those sweep cells), 32-row tiles otherwise
+        const bool small_tiles = 4 * pl->k >= L || (L >= 128 && 8 * pl->k >= L);
+        const Cand pr[] = {{LAGKV_TUNE_PAIRS, small_tiles ? 16 : 32, 2, 1}, {LAGKV_TUNE_PAIRS, small_tiles ? 32 : 16, 2, 1}};
         Shape sh;
         rc = first_fit(pl, pr, 2, &sh);
         if (rc == LAGKV_ECUDA) return rc;
