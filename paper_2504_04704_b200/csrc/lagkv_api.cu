@@ -132,10 +132,16 @@ int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Sha
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
     if (smem > size_t(pl->max_smem_optin)) return LAGKV_EUNSUPPORTED;
     if ((smem + 1024) * size_t(ctas) > size_t(kSmemPerSm)) return LAGKV_EUNSUPPORTED;
-    if (pl->cfg.device >= 0 &&
-        cudaFuncSetAttribute(reinterpret_cast<const void*>(kKernels[kidx].fn),
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-        return LAGKV_ECUDA;
+    if (pl->cfg.device >= 0) {
+        // the limit belongs to the function, not to the plan: only ever raise it, so that shapes of
+        // the same kernel with deeper rings (this plan's or another's) keep launching
+        const void* fn = reinterpret_cast<const void*>(kKernels[kidx].fn);
+        cudaFuncAttributes attr;
+        if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return LAGKV_ECUDA;
+        if (size_t(attr.maxDynamicSharedSizeBytes) < smem &&
+            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+            return LAGKV_ECUDA;
+    }
     out->kidx = kidx;
     out->stages = stages;
     out->ctas_per_sm = ctas;
@@ -161,7 +167,7 @@ int first_fit(const lagkv_plan_s* pl, const Cand* cands, int nc, Shape* out) {
 // CTA per (b, h).
 int choose_shape(lagkv_plan_s* pl) {
     const int L = pl->cfg.lag;
-    Cand uni[10];
+    Cand uni[8];
     int nu = 0;
     if (L >= 1024 && pl->cfg.variant == LAGKV_VARIANT_LAGKV) {  // eight-warp CTAs are compiled for LagKV only
         uni[nu++] = {8, 32, 3, 1};
@@ -171,14 +177,18 @@ int choose_shape(lagkv_plan_s* pl) {
         uni[nu++] = {4, 32, 3, 2};
         uni[nu++] = {4, 32, 2, 2};
     }
-    uni[nu++] = {2, 16, 2, 6};  // two stages: 3-4 % ahead of three on the short-partition sweep cells
+    const int two_warp = nu;
     uni[nu++] = {2, 16, 3, 6};
     uni[nu++] = {2, 16, 3, 4};
     uni[nu++] = {2, 16, 2, 2};
     uni[nu++] = {2, 16, 2, 1};
-    int rc = first_fit(pl, uni, nu, &pl->app);
+    int rc = first_fit(pl, uni, nu, &pl->app);  // appends: deeper rings also mean larger chunks for the in-place move
     if (rc != LAGKV_OK) return rc;
     pl->pre = pl->app;
+    if (two_warp == 0) {  // short partitions, prefill: two stages are 3-4 % ahead of three on the sweep cells
+        Shape sh;
+        if (make_shape(pl, 2, 16, 2, 6, &sh) == LAGKV_OK) pl->pre = sh;
+    }
     pl->pair.kidx = -1;
     pl->tuned = false;
     if (L >= 256) {

@@ -942,6 +942,33 @@ def test_bounded_wait_gives_up_and_reports(binding):
     assert plan.read_status(ws)[0] == 0 and out["L_R"] == 4 + 2 * 16 + 64
 
 
+def test_plans_do_not_lower_each_others_limits(binding, oracle):
+    """The dynamic shared memory limit is a property of the kernel function: a later plan that
+    needs less (shorter partitions, shallower rings) must not stop an earlier plan's launches."""
+    B, H, D, sink = 1, 2, 128, 16
+    big = binding.Plan(B, H, D, sink, 2048, keep_k=256, device=0)
+    small = binding.Plan(B, H, D, sink, 256, keep_k=64, device=0)          # same kernel, less shared memory
+    for plan, L, k in ((big, 2048, 256), (small, 256, 64), (big, 2048, 256)):
+        S = sink + 3 * L + 50
+        K, V = synth.make_kv(B, H, S, D, seed=L, device="cuda:0")
+        ws = plan.new_workspace()
+        out = plan.compress_prefill(K, V, ws)
+        assert plan.read_status(ws)[0] == 0
+        ref = oracle.compress(synth.to_bits(K), synth.to_bits(V), sink, L, k, want_scores=False)
+        np.testing.assert_array_equal(synth.to_bits(out["K_out"]), np.take_along_axis(
+            synth.to_bits(K), out["idx"].cpu().numpy()[..., None].astype(np.int64), axis=2))
+        assert out["L_R"] == ref["L_R"]
+    # appends (three-stage rings) after a prefill plan of the same kernel with two stages
+    a = binding.Plan(2, 2, D, 8, 96, keep_k=24, device=0)
+    binding.Plan(2, 2, D, 8, 64, keep_k=16, device=0)
+    Kc, Vc = synth.make_kv(2, 2, 8 + 3 * 96 + 20, D, seed=3, device="cuda:0")
+    seq = torch.tensor([8 + 2 * 96 + 5, 8 + 3 * 96], dtype=torch.int32, device="cuda:0")
+    stat = torch.full((2,), 8, dtype=torch.int32, device="cuda:0")
+    wsa = a.new_workspace(2)
+    a.compress_append(Kc, Vc, seq, stat, wsa, max_new_chunks=2)
+    assert a.read_status(wsa)[0] == 0 and stat.tolist() == [8 + 24, 8 + 48]
+
+
 # ----------------------------------------------------------------------- argument checks
 def test_argument_errors(binding):
     with pytest.raises(binding.LagKVError) as e:
