@@ -136,6 +136,8 @@ int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Sha
         // the limit belongs to the function, not to the plan: only ever raise it, so that shapes of
         // the same kernel with deeper rings (this plan's or another's) keep launching
         const void* fn = reinterpret_cast<const void*>(kKernels[kidx].fn);
+        static std::mutex limit_mu;  // read-then-raise must not interleave between threads
+        std::lock_guard<std::mutex> lock(limit_mu);
         cudaFuncAttributes attr;
         if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return LAGKV_ECUDA;
         if (size_t(attr.maxDynamicSharedSizeBytes) < smem &&
