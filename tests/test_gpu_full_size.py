@@ -162,3 +162,60 @@ def test_full_size_decode_append(binding, oracle):
         np.testing.assert_array_equal(synth.to_bits(K[b:b + 1, :, :m]), Kb[:, :, :m])
         np.testing.assert_array_equal(synth.to_bits(V[b:b + 1, :, :m]), Vb[:, :, :m])
     print(f"decode_append: {calls} calls, {triggers} triggers, {len(sample)} sequences replayed by the oracle")
+
+
+def test_full_size_decode_append_ragged(binding, oracle):
+    """Config 3 with per-sequence window offsets: the 448 (sequence, layer) caches start with
+    windows of different fill, so every call of the append entry point compresses some sequences
+    and skips the others.  1024 tokens are appended in blocks of 64; sampled sequences are
+    replayed by the oracle, and the number of compressions is the one the lengths imply."""
+    w = synth.WORKLOADS["decode_append"]
+    Bf, H, D, L, sink = w.layers * w.B, w.H, w.D, w.lag, w.sink
+    plan = binding.Plan(Bf, H, D, sink, L, keep_ratio=w.ratio, device=0)
+    k = plan.k
+    stat0, grow, block = sink + 123 * k, 1024, 64
+    fill = (torch.arange(Bf, dtype=torch.int64) * 37) % L                 # rows beyond one full partition
+    start = stat0 + L + fill                                              # stored rows per sequence
+    S_cap = int(start.max()) + grow + 8
+    K = torch.empty((Bf, H, S_cap, D), dtype=torch.bfloat16, device="cuda:0")
+    V = torch.empty_like(K)
+    for layer in range(w.layers):
+        sl = slice(layer * w.B, (layer + 1) * w.B)
+        K[sl], V[sl] = synth.make_kv(w.B, H, S_cap, D, w.seed(layer) + 500, device="cuda:0")
+    # rows [start_b + t] of the initial buffers are the tokens appended later: keep a copy of them
+    idx_new = (start[:, None] + torch.arange(grow)[None, :]).to("cuda:0")                  # [Bf, grow]
+    take = idx_new[:, None, :, None].expand(Bf, H, grow, D)
+    Knew, Vnew = torch.gather(K, 2, take), torch.gather(V, 2, take)
+    seq = start.to(torch.int32).to("cuda:0")
+    stat = torch.full((Bf,), stat0, dtype=torch.int32, device="cuda:0")
+    ws = plan.new_workspace(1)
+    rng = np.random.default_rng(5)
+    sample = sorted({0, Bf - 1, *map(int, rng.integers(Bf, size=4))})
+    ref = {b: (synth.to_bits(K[b:b + 1]), synth.to_bits(V[b:b + 1]), np.array([int(start[b])]), np.array([stat0]))
+           for b in sample}
+    bidx = torch.arange(Bf, device="cuda:0")
+    triggers = 0
+    for done in range(0, grow, block):
+        pos = seq.long()[:, None] + torch.arange(block, device="cuda:0")[None, :]          # where the new rows go
+        K[bidx[:, None], :, pos] = Knew[:, :, done:done + block].permute(0, 2, 1, 3)
+        V[bidx[:, None], :, pos] = Vnew[:, :, done:done + block].permute(0, 2, 1, 3)
+        seq += block
+        before = stat.clone()
+        plan.compress_append(K, V, seq, stat, ws, max_new_chunks=1)
+        triggers += int((stat != before).sum())
+        for b in sample:
+            Kb, Vb, sb, tb = ref[b]
+            c = int(sb[0])
+            Kb[:, :, c:c + block] = synth.to_bits(Knew[b:b + 1, :, done:done + block])
+            Vb[:, :, c:c + block] = synth.to_bits(Vnew[b:b + 1, :, done:done + block])
+            ref[b] = oracle.compress_append(Kb, Vb, sb + block, tb, L, k)[:4]
+    assert plan.read_status(ws)[0] == 0
+    want = int(((L + fill + grow) // L - 1).sum())                        # partitions completed per sequence
+    assert triggers == want and 0 < triggers
+    for b in sample:
+        Kb, Vb, sb, tb = ref[b]
+        m = int(sb[0])
+        assert int(seq[b]) == m and int(stat[b]) == int(tb[0])
+        np.testing.assert_array_equal(synth.to_bits(K[b:b + 1, :, :m]), Kb[:, :, :m])
+        np.testing.assert_array_equal(synth.to_bits(V[b:b + 1, :, :m]), Vb[:, :, :m])
+    print(f"decode_append ragged: {grow // block} calls, {triggers} compressions over {Bf} sequences")
