@@ -2,6 +2,8 @@
 """Benchmark of the LagKV prefill compress pass on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+                    [--variant lagkv|localkv|l2norm] [--storage bf16|fp16] [--layers N] [--tune w,t,s,c]
+    python bench.py --workload decode_append --append        # the incremental pass, one call per step
 
 A step is one whole compress pass (partition, lag statistics, normalise + std, softmax,
 K+V sum, per-head top-k, compaction, sink and window copy) over every layer of one
