@@ -26,7 +26,12 @@
  *     Errors detected on the host leave all buffers untouched.  Errors detected on the
  *     device (a bounded wait that ran out, an append that would overflow idx capacity)
  *     are recorded in the status block at the start of the workspace and reported by
- *     lagkv_read_status(); the kernels never trap or spin forever.
+ *     lagkv_read_status(); the kernels never trap or spin forever.  After LAGKV_ETIMEOUT
+ *     the outputs of that call are incomplete: a prefill's K_out / V_out / idx_out hold
+ *     undefined rows; an append leaves seq_len / static_len of every sequence one of whose
+ *     heads gave up as they were before the call, and the rows of such a sequence behind
+ *     its static part are undefined (other heads may already have been moved).  The
+ *     workspace itself stays usable: the per-sequence counters return to zero.
  *   - The workspace is caller-owned device memory of at least lagkv_workspace_bytes()
  *     bytes, 256-byte aligned, cleared once with lagkv_workspace_init() and then reusable
  *     across calls on the same stream.  Calls sharing a workspace must not overlap.
@@ -58,7 +63,10 @@ enum lagkv_variant {
     LAGKV_VARIANT_LAGKV = 0,   /* Eq. 7-11: statistics from the next partition        */
     LAGKV_VARIANT_LOCALKV = 1, /* Eq. 14, Eq. 15: statistics from the partition itself */
     LAGKV_VARIANT_L2NORM = 2   /* Eq. 16: score = -||K row||_2, no softmax, V is only
-                                  gathered                                             */
+                                  gathered.  Section 4.3 leaves the first two layers of
+                                  the model uncompressed for this variant: layers have
+                                  no dimension here, so the caller keeps those two
+                                  layers out of the batch it folds into B               */
 };
 
 enum lagkv_dtype {
@@ -103,6 +111,15 @@ int32_t lagkv_keep_count(lagkv_plan_t plan);
  * bullet of Section 2.2).  Pure host arithmetic.  static_len < 0 means "the plan's sink".
  */
 int64_t lagkv_compressed_len(lagkv_plan_t plan, int64_t seq_len, int64_t static_len);
+
+/*
+ * The two lengths of a sequence after a pass (Section 2.2, bullets 2-4; Eq. 12): what
+ * lagkv_compress_append() writes to seq_len[b] and static_len[b] on the device, computed on the
+ * host so that a driver loop can mirror them without a read-back.  rest < 2L: both unchanged.
+ * static_len < 0 means "the plan's sink".  Returns LAGKV_EINVAL for seq_len < static_len.
+ */
+int lagkv_lengths_after(lagkv_plan_t plan, int64_t seq_len, int64_t static_len, int64_t *new_seq_len,
+                        int64_t *new_static_len);
 
 /*
  * Inverse of Eq. 12 / Eq. 13 as used for the adaptive retention ratio of Section 3.2:
@@ -205,6 +222,10 @@ int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64
  *   status_out  DEVICE int32[4] or NULL: receives the status block of this call (same
  *               meaning as lagkv_read_status(): [0] first device-side status, [1] detail,
  *               [2] zero-range channel count), written on cuda_stream after the kernels.
+ *               With NULL the block stays in the built-in array until the next call on that
+ *               device clears it: read it before then with lagkv_read_status(plan, NULL, ...),
+ *               or a device-side LAGKV_ECAPACITY / LAGKV_EINVAL / LAGKV_ETIMEOUT of this call
+ *               goes unnoticed.
  * The call allocates nothing and frees nothing; it enqueues a small memset (status block and
  * counters), the append kernel and, if asked, a 16-byte device-to-device copy.
  *
@@ -241,7 +262,9 @@ int lagkv_gather(lagkv_plan_t plan, const void *K, const void *V, int64_t S_in,
                  void *cuda_stream);
 
 /*
- * Synchronise cuda_stream, copy the status block to the host and clear it.
+ * Synchronise cuda_stream, copy the status block to the host and clear it.  workspace == NULL
+ * names the status block of the library's built-in scratch on the plan's device (the one
+ * lagkv_compress_append_noalloc() uses).
  * host_status[0] = first device-side lagkv_status recorded since the last read (0 = none),
  * host_status[1] = detail (block index), host_status[2] = count of zero-range reference
  * channels seen, host_status[3] = reserved.  Returns host_status[0], or LAGKV_ECUDA.

@@ -27,7 +27,7 @@ VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
 # every symbol include/lagkv.h declares
 EXPORTS = (
     "lagkv_plan", "lagkv_plan_destroy", "lagkv_keep_count", "lagkv_compressed_len",
-    "lagkv_keep_for_target", "lagkv_workspace_bytes", "lagkv_workspace_init",
+    "lagkv_keep_for_target", "lagkv_lengths_after", "lagkv_workspace_bytes", "lagkv_workspace_init",
     "lagkv_compress_prefill", "lagkv_compress_prefill_host", "lagkv_host_staging_bytes",
     "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
     "lagkv_read_status",
@@ -74,6 +74,8 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_keep_count.argtypes = [vp]
     lib.lagkv_compressed_len.restype = i64
     lib.lagkv_compressed_len.argtypes = [vp, i64, i64]
+    lib.lagkv_lengths_after.restype = ctypes.c_int
+    lib.lagkv_lengths_after.argtypes = [vp, i64, i64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.lagkv_keep_for_target.restype = i32
     lib.lagkv_keep_for_target.argtypes = [i64, i32, i32, ctypes.c_double]
     lib.lagkv_workspace_bytes.restype = sz
@@ -171,6 +173,13 @@ class Plan:
     def compressed_len(self, seq_len: int, static_len: int = -1) -> int:
         return int(self.lib.lagkv_compressed_len(self.handle, int(seq_len), int(static_len)))
 
+    def lengths_after(self, seq_len: int, static_len: int = -1) -> tuple[int, int]:
+        """``lagkv_lengths_after``: (seq_len, static_len) of a sequence after one pass."""
+        a, b = ctypes.c_int64(), ctypes.c_int64()
+        _check(self.lib.lagkv_lengths_after(self.handle, int(seq_len), int(static_len), ctypes.byref(a),
+                                            ctypes.byref(b)), "lagkv_lengths_after")
+        return int(a.value), int(b.value)
+
     def workspace_bytes(self, max_new_chunks: int = 0) -> int:
         return int(self.lib.lagkv_workspace_bytes(self.handle, int(max_new_chunks)))
 
@@ -194,7 +203,8 @@ class Plan:
                "lagkv_workspace_init")
         return ws
 
-    def read_status(self, workspace: torch.Tensor) -> list[int]:
+    def read_status(self, workspace) -> list[int]:
+        """``lagkv_read_status``; ``workspace=None`` reads the library's built-in scratch."""
         st = (ctypes.c_int32 * 4)()
         rc = self.lib.lagkv_read_status(self.handle, _ptr(workspace), _stream(self._dev()), ctypes.byref(st))
         if rc == LAGKV_ECUDA or rc == LAGKV_EINVAL and st[0] != LAGKV_EINVAL:
@@ -319,36 +329,47 @@ class ChunkedPrefill:
     appends them to the caches held here and runs the append pass, so the caches never grow
     beyond ``capacity`` rows.  All sequences advance together."""
 
-    def __init__(self, B, H_kv, D, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1, capacity=None, device=0):
-        self.plan = Plan(B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof, device=device)
+    def __init__(self, B, H_kv, D, sink, lag, keep_ratio=0.25, keep_k=0, std_ddof=1, capacity=None, device=0,
+                 variant=VARIANT_LAGKV, dtype=torch.bfloat16):
+        self.plan = Plan(B, H_kv, D, sink, lag, keep_ratio=keep_ratio, keep_k=keep_k, std_ddof=std_ddof, device=device,
+                         variant=variant, dtype=dtype)
         dev = self.plan._dev()
         self.first = sink + 2 * lag                     # tokens of the first step
         self.step = lag                                 # tokens of every later step
         self.capacity = int(capacity if capacity is not None else sink + 4 * lag)
-        self.K = torch.zeros((B, H_kv, self.capacity, D), dtype=torch.bfloat16, device=dev)
+        self.K = torch.zeros((B, H_kv, self.capacity, D), dtype=dtype, device=dev)
         self.V = torch.zeros_like(self.K)
         self.seq_len = torch.zeros((B,), dtype=torch.int32, device=dev)
         self.static_len = torch.full((B,), sink, dtype=torch.int32, device=dev)
         self.ws = self.plan.new_workspace(2)
-        self.rows = 0                                   # stored rows (host copy of seq_len, all equal)
-        self.static = sink
+        self.rows = 0                                   # stored rows (host mirror of seq_len, all equal)
+        self.static = sink                              # host mirror of static_len
 
-    def feed(self, K_new, V_new) -> None:
-        """Append ``[B, H, t, D]`` new rows (any t that fits) and compress."""
+    def feed(self, K_new, V_new, check_status: bool = False) -> None:
+        """Append ``[B, H, t, D]`` new rows (any t that fits) and compress.  The host mirrors of
+        the two lengths come from the library (``lagkv_lengths_after``), so no read-back is
+        needed between steps; ``check_status`` synchronises and raises on a device-side error
+        (without it, call ``status()`` at the end of the prompt)."""
         t = int(K_new.shape[2])
         if self.rows + t > self.capacity:
             raise ValueError("chunk does not fit the cache capacity")
+        # more partitions than the workspace was sized for would be refused on the device
+        if (self.rows + t - self.static) // self.plan.cfg.lag - 1 > 2:
+            raise ValueError("chunk completes more than two partitions at once")
         self.K[:, :, self.rows:self.rows + t] = K_new
         self.V[:, :, self.rows:self.rows + t] = V_new
         self.seq_len += t
         self.rows += t
         self.plan.compress_append(self.K, self.V, self.seq_len, self.static_len, self.ws, max_new_chunks=2)
-        # the same integers on the host (Eq. 12): no device read-back needed between steps
-        new_rows = self.plan.compressed_len(self.rows, self.static)
-        rest = self.rows - self.static
-        if rest >= 2 * self.plan.cfg.lag:
-            self.static += (rest // self.plan.cfg.lag - 1) * self.plan.k
-        self.rows = new_rows
+        self.rows, self.static = self.plan.lengths_after(self.rows, self.static)
+        if check_status:
+            self.status()
+
+    def status(self) -> None:
+        """Synchronise and raise if any append since the last check recorded a device-side error."""
+        st = self.plan.read_status(self.ws)
+        if st[0] != LAGKV_OK:
+            raise LagKVError(st[0], "lagkv_compress_append (device status)")
 
 
 class HostPrefill:

@@ -241,6 +241,34 @@ int check_launch() {
 
 }  // namespace
 
+// ------------------------------------------------------------------ append without a workspace
+// Scratch that lagkv_compress_append_noalloc() hands to the append kernel in place of a
+// caller-supplied workspace: the 256-byte status block followed by the kept-position list.
+// It lives in the library image, one copy per GPU that loads the library, until the process
+// exits.  In host code the symbol below is only a handle: the address a kernel can use comes
+// from cudaGetSymbolAddress(), asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LAGKV_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device` (which must be current); nullptr on error.
+void* noalloc_scratch_for(int device) {
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[device] == nullptr) {
+        int current = -1;  // the lookup answers for the CURRENT device: never cache it under another ordinal
+        if (cudaGetDevice(&current) != cudaSuccess || current != device) return nullptr;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
+        g_noalloc_ptr[device] = ptr;
+    }
+    return g_noalloc_ptr[device];
+}
+}  // namespace
+
 extern "C" {
 
 int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
@@ -255,7 +283,7 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
     if (cfg->dtype != LAGKV_DTYPE_BF16 && cfg->dtype != LAGKV_DTYPE_FP16) return LAGKV_EINVAL;
     if (cfg->D != 64 && cfg->D != 96 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
-    if ((long long)cfg->B * cfg->H_kv > (1ll << 30)) return LAGKV_EINVAL;
+    if ((long long)cfg->B * cfg->H_kv > (1ll << 30) || cfg->H_kv >= kSeqFailed) return LAGKV_EINVAL;
 
     lagkv_plan_s* pl = new (std::nothrow) lagkv_plan_s();
     if (pl == nullptr) return LAGKV_EINVAL;
@@ -290,6 +318,22 @@ int64_t lagkv_compressed_len(lagkv_plan_t plan, int64_t seq_len, int64_t static_
     const int64_t rest = seq_len - st;
     if (rest < 2 * L) return seq_len;
     return st + int64_t(plan->k) * (rest / L - 1) + L + rest % L;
+}
+
+int lagkv_lengths_after(lagkv_plan_t plan, int64_t seq_len, int64_t static_len, int64_t* new_seq_len,
+                        int64_t* new_static_len) {
+    if (plan == nullptr || new_seq_len == nullptr || new_static_len == nullptr) return LAGKV_EINVAL;
+    const int64_t L = plan->cfg.lag, st = static_len < 0 ? plan->cfg.sink : static_len;
+    const int64_t rest = seq_len - st;
+    if (rest < 0) return LAGKV_EINVAL;
+    if (rest < 2 * L) {  // third bullet of Section 2.2: nothing happens
+        *new_seq_len = seq_len;
+        *new_static_len = st;
+        return LAGKV_OK;
+    }
+    *new_static_len = st + int64_t(plan->k) * (rest / L - 1);
+    *new_seq_len = *new_static_len + L + rest % L;
+    return LAGKV_OK;
 }
 
 int32_t lagkv_keep_for_target(int64_t Ls, int32_t sink, int32_t lag, double target_C) {
@@ -516,9 +560,11 @@ int lagkv_compress_prefill_host(lagkv_plan_t plan, const void* K_host, const voi
     return ok ? LAGKV_OK : LAGKV_ECUDA;
 }
 
-int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
-                          int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
-                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// Host-side checks of an append call (everything that can be refused before any stream work).
+static int append_check(lagkv_plan_t plan, const void* K_cache, const void* V_cache, int64_t S_cap,
+                        const int32_t* seq_len, const int32_t* static_len, int32_t max_new_chunks,
+                        const int32_t* idx_out, const float* scores_out, const void* workspace,
+                        size_t workspace_bytes, Strides* st) {
     if (plan == nullptr || K_cache == nullptr || V_cache == nullptr || seq_len == nullptr || static_len == nullptr ||
         plan->cfg.device < 0)
         return LAGKV_EINVAL;
@@ -532,9 +578,18 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     const size_t head = (kStatusWords + counter_words(plan)) * sizeof(int32_t);
     const size_t need = idx_out ? head : lagkv_workspace_bytes(plan, max_new_chunks);
     if (workspace_bytes < need) return LAGKV_EWORKSPACE;
-    const lagkv_config& c = plan->cfg;
+    if (resolve_strides(plan->cfg, S_cap, st) != LAGKV_OK) return LAGKV_EINVAL;
+    return LAGKV_OK;
+}
+
+int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
+                          int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
     Strides st;
-    if (resolve_strides(c, S_cap, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    const int chk = append_check(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out,
+                                 scores_out, workspace, workspace_bytes, &st);
+    if (chk != LAGKV_OK) return chk;
+    const lagkv_config& c = plan->cfg;
 
     DeviceGuard guard(c.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -601,9 +656,12 @@ int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, 
 }
 
 int lagkv_read_status(lagkv_plan_t plan, void* workspace, void* cuda_stream, int32_t host_status[4]) {
-    if (plan == nullptr || workspace == nullptr || host_status == nullptr || plan->cfg.device < 0)
-        return LAGKV_EINVAL;
+    if (plan == nullptr || host_status == nullptr || plan->cfg.device < 0) return LAGKV_EINVAL;
     DeviceGuard guard(plan->cfg.device);
+    if (workspace == nullptr) {  // the status block of the library's built-in scratch on the plan's device
+        workspace = noalloc_scratch_for(plan->cfg.device);
+        if (workspace == nullptr) return LAGKV_ECUDA;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemcpyAsync(host_status, workspace, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return LAGKV_ECUDA;
@@ -685,32 +743,6 @@ const char* lagkv_version(void) { return "lagkv-b200 0.1 (sm_100a)"; }
 
 }  // extern "C"
 
-// ------------------------------------------------------------------ append without a workspace
-// Scratch that lagkv_compress_append_noalloc() hands to the append kernel in place of a
-// caller-supplied workspace: the 256-byte status block followed by the kept-position list.
-// It lives in the library image, one copy per GPU that loads the library, until the process
-// exits.  In host code the symbol below is only a handle: the address a kernel can use comes
-// from cudaGetSymbolAddress(), asked once per device with that device current.
-static __device__ __align__(256) unsigned char g_noalloc_scratch[LAGKV_NOALLOC_SCRATCH_BYTES];
-
-namespace {
-constexpr int kMaxDevices = 64;
-std::mutex g_noalloc_mutex;
-void* g_noalloc_ptr[kMaxDevices] = {};
-
-// Device address of the scratch array on `device` (which must be current); nullptr on error.
-void* noalloc_scratch_for(int device) {
-    if (device < 0 || device >= kMaxDevices) return nullptr;
-    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
-    if (g_noalloc_ptr[device] == nullptr) {
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
-        g_noalloc_ptr[device] = ptr;
-    }
-    return g_noalloc_ptr[device];
-}
-}  // namespace
-
 extern "C" int lagkv_compress_append_noalloc(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap,
                                              int32_t* seq_len, int32_t* static_len, int32_t max_new_chunks,
                                              int32_t* idx_out, float* scores_out, int32_t* status_out,
@@ -725,6 +757,12 @@ extern "C" int lagkv_compress_append_noalloc(lagkv_plan_t plan, void* K_cache, v
     void* scratch = noalloc_scratch_for(plan->cfg.device);
     if (scratch == nullptr) return LAGKV_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    {  // refuse bad arguments before anything is enqueued: a refused call leaves the scratch as it was
+        Strides st;
+        const int chk = append_check(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out,
+                                     scores_out, scratch, size_t(LAGKV_NOALLOC_SCRATCH_BYTES), &st);
+        if (chk != LAGKV_OK) return chk;
+    }
     // the array keeps what the previous call left: the status block and the per-sequence head
     // counters have to start at zero
     if (cudaMemsetAsync(scratch, 0, head, stream) != cudaSuccess) return LAGKV_ECUDA;

@@ -16,7 +16,7 @@
 //   * At the end of a partition the CTA runs softmax over the L tokens for K and V, adds
 //     them (Eq. 11), selects the k best with a radix select on the fp32 bit pattern
 //     (ties to the lower index) and copies the kept rows straight to the output layout
-//     (rows come back from L2, which they passed through moments before).
+//     (a second read: by then the rows have left L2 again and come from DRAM).
 //
 // No tensor cores: the pass is a streaming reduction / selection / gather.
 #pragma once
@@ -27,6 +27,7 @@ namespace lagkv {
 
 constexpr int kStatusWords = 64;  // 256-byte status block at the start of the workspace
 constexpr int kMaxWarps = 16;
+constexpr int kSeqFailed = 1 << 24;  // added to a sequence's head counter by a head that gave up (H_kv < 2^24)
 
 enum { MODE_PREFILL = 0, MODE_APPEND = 1 };
 enum { ST_OK = 0, ST_EINVAL = 1, ST_ETIMEOUT = 5, ST_ECAPACITY = 6 };
@@ -1198,13 +1199,13 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     }
 
     // ---- append: pack kept rows behind the static part, then slide the window down
-    if (P.mode == MODE_APPEND && !aborted) {
+    if (P.mode == MODE_APPEND) {
         const int u = unit_fixed;
         uint16_t* ck = const_cast<uint16_t*>(unit_base(P.K, u));
         uint16_t* cv = const_cast<uint16_t*>(unit_base(P.V, u));
         const int n_c = n - 1;
         const int32_t* kp = P.kept_pos + (long long)u * P.max_chunks * k;
-        if (k < L && warp == 0) {  // kept rows, then the window, as one ascending sequence of rows
+        if (!aborted && k < L && warp == 0) {  // kept rows, then the window, as one ascending sequence of rows
             const int R = int(smem_ring_bytes<G>(NS) / (4 * G::D * 2));
             if (!move_rows_bulk<G>(ck, cv, P.ss, stat_rows, n_c * k + L + rem, n_c * k, kp,
                                    stat_rows + n_c * L - n_c * k, smem_u32(ring), R, smem_u32(move_bars), lane)) {
@@ -1214,14 +1215,20 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         }
         // The lengths of a sequence change once all of its heads are done: every head's CTA has
         // read the old values by then.  The last one to finish writes the new ones and clears
-        // the counter for the next call.
+        // the counter for the next call.  A head whose wait ran out still counts (so that the
+        // counter returns to zero) and marks the sequence as failed: its lengths stay as they
+        // were, and its rows after the static part are undefined.
         if (tid == 0) {
             const int b = u / P.H;
-            if (atomicAdd(P.seq_done + b, 1) == P.H - 1) {
+            const bool failed = aborted || timed_out;  // tid 0 sits in warp 0, which did the move
+            const int old = atomicAdd(P.seq_done + b, failed ? 1 + kSeqFailed : 1);
+            if ((old & (kSeqFailed - 1)) == P.H - 1) {
                 P.seq_done[b] = 0;
-                const int ns = stat_rows + n_c * k;
-                const_cast<int32_t*>(P.static_len)[b] = ns;
-                const_cast<int32_t*>(P.seq_len)[b] = ns + L + rem;
+                if (!failed && old < kSeqFailed) {
+                    const int ns = stat_rows + n_c * k;
+                    const_cast<int32_t*>(P.static_len)[b] = ns;
+                    const_cast<int32_t*>(P.seq_len)[b] = ns + L + rem;
+                }
             }
         }
     }

@@ -33,6 +33,7 @@ __host__ __device__ inline size_t pair_smem_total_bytes(int stages, int L) {
     s += size_t(G::NW) * 2 * (G::D / 2) * 4;           // own min / max row of every streaming warp
     s += size_t(kPairs) * 2 * 2 * Lp * 4;              // sigma [pair][2 buffers][K, V]
     s += size_t(kPairs) * Lp * 4;                      // kept indices [pair]
+    s += size_t(kPairs) * 4;                           // give-up flag [pair]
     return s + 128;                                    // alignment slack
 }
 
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
     float* sgbase = reinterpret_cast<float*>(stats + G::NW * 2 * STAT_WORDS);
     const int Lp = (P.L + 3) & ~3;
     int* keptbase = reinterpret_cast<int*>(sgbase + kPairs * 4 * Lp);
+    volatile int* gave_up = reinterpret_cast<volatile int*>(keptbase + kPairs * Lp);  // [pair]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = P.L, k = P.k, n = P.n, sink = P.sink;
@@ -180,6 +182,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             mbar_init(full_bar + 8 * b, 2);   // the K warp and the V warp
             mbar_init(empty_bar + 8 * b, 1);  // the epilogue warp
         }
+        gave_up[pair] = 0;
     }
     fence_mbar_init();
     fence_proxy_async();
@@ -190,9 +193,15 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
     };
     float* sg_pair = sgbase + pair * 4 * Lp;  // [2 buffers][K, V][Lp]
     bool dead = false;
+    // A warp whose wait ran out stops working, raises its pair's flag (the sigma values it owes
+    // are incomplete, so the pair's epilogue warp must not select or emit from them any more)
+    // and keeps only its arrivals alive.
     auto give_up = [&]() {  // warp-collective
         dead = true;
-        if (lane == 0) record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+        if (lane == 0) {
+            record_status(P.status, ST_ETIMEOUT, blockIdx.x);
+            gave_up[pair] = 1;
+        }
     };
 
     if (streamer) {
@@ -327,6 +336,8 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             const bool top = p == n - 1;
             const bool score = !top && s >= s_first;
             if (!dead && !mbar_wait_bounded(full_bar + 8 * buf, uint32_t(i >> 1) & 1u)) give_up();
+            // the flag is raised before the arrival that completes the phase waited for above
+            if (!dead && __shfl_sync(0xffffffffu, gave_up[pair], 0) != 0) dead = true;
             const uint32_t ebar = empty_bar + 8 * buf;
             const uint16_t* uk = unit_base(P.K, u);
             const uint16_t* uv = unit_base(P.V, u);

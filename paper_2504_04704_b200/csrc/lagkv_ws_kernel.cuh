@@ -465,9 +465,19 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     // memory system.
     __syncthreads();
     if (P.K_out != nullptr && *abort_flag == 0) {
-        constexpr int NTALL = G::NT + kWsEpiWarps * 32;
-        constexpr int U = 8;
-        const int items = k * 2 * G::VPR;  // 32 consecutive items = one kept row of K and of V
+        constexpr int NWALL = G::NW + kWsEpiWarps;
+        // A kept row is 2 * VPR 16-byte vectors (K, then V).  A warp always moves WHOLE rows, GR at
+        // a time (the smallest count whose vectors fill the 32 lanes evenly, IPL per lane), UG
+        // such groups per pass so that 6-8 loads are in flight per lane.  Without idx_out the
+        // position of a kept row is parked in the first word of its K_out row: because the warp
+        // that reads that word is the only one that ever writes the row, reading all positions
+        // of a pass before its first store (warp barrier below) is enough for every head_dim.
+        constexpr int RV = 2 * G::VPR;
+        constexpr int GR = (RV % 32 == 0) ? 1 : ((RV % 16 == 0) ? 2 : 4);
+        constexpr int IPL = GR * RV / 32;
+        constexpr int UG = IPL == 1 ? 8 : (IPL == 2 ? 4 : 2);
+        static_assert((GR * RV) % 32 == 0 && IPL * 32 == GR * RV, "a row group must fill the warp evenly");
+        const int ngroups = (k + GR - 1) / GR;
         // slots the copy warp claimed are done; the rest (at least the last one) is moved here
         const long long s_from = s_lo + *reinterpret_cast<volatile int*>(&sc.claimed);
         for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
@@ -478,36 +488,41 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             const long long o = (long long)u * P.L_R + sink + p * k;
             uint16_t* dstK = P.K_out + o * G::D;
             uint16_t* dstV = P.V_out + o * G::D;
-            for (int base = 0; base < items; base += NTALL * U) {
-                int src[U];
-                uint4 buf[U];
+            for (int g0 = warp; g0 < ngroups; g0 += NWALL * UG) {
+                int src[UG][IPL];
+                uint4 buf[UG][IPL];
 #pragma unroll
-                for (int q = 0; q < U; ++q) {
-                    const int i = base + q * NTALL + tid;
-                    if (i < items) {
-                        const int j = (i / G::VPR) >> 1;
-                        src[q] = P.idx_out != nullptr ? __ldcg(P.idx_out + o + j)
-                                                      : __ldcg(reinterpret_cast<const int32_t*>(dstK + (long long)j * G::D));
-                    }
-                }
+                for (int q = 0; q < UG; ++q)
 #pragma unroll
-                for (int q = 0; q < U; ++q) {
-                    const int i = base + q * NTALL + tid;
-                    if (i < items) {
-                        const int vec = i % G::VPR, r2 = i / G::VPR;
-                        const uint16_t* sp = (r2 & 1) ? srcV : srcK;
-                        buf[q] = ld_nc(reinterpret_cast<const uint4*>(sp + (long long)src[q] * P.ss) + vec);
+                    for (int e = 0; e < IPL; ++e) {
+                        const int j = (g0 + q * NWALL) * GR + (e * 32 + lane) / RV;
+                        src[q][e] = -1;
+                        if (g0 + q * NWALL < ngroups && j < k)
+                            src[q][e] = P.idx_out != nullptr
+                                            ? __ldcg(P.idx_out + o + j)
+                                            : __ldcg(reinterpret_cast<const int32_t*>(dstK + (long long)j * G::D));
                     }
-                }
+                __syncwarp();  // every parked position of this pass is read before a row is overwritten
 #pragma unroll
-                for (int q = 0; q < U; ++q) {
-                    const int i = base + q * NTALL + tid;
-                    if (i < items) {
-                        const int vec = i % G::VPR, r2 = i / G::VPR, j = r2 >> 1;
-                        uint16_t* dp = (r2 & 1) ? dstV : dstK;
-                        st_stream(reinterpret_cast<uint4*>(dp + (long long)j * G::D) + vec, buf[q]);
-                    }
-                }
+                for (int q = 0; q < UG; ++q)
+#pragma unroll
+                    for (int e = 0; e < IPL; ++e)
+                        if (src[q][e] >= 0) {
+                            const int va = (e * 32 + lane) % RV;
+                            const uint16_t* sp = va >= G::VPR ? srcV : srcK;
+                            buf[q][e] = ld_nc(reinterpret_cast<const uint4*>(sp + (long long)src[q][e] * P.ss) +
+                                              (va % G::VPR));
+                        }
+#pragma unroll
+                for (int q = 0; q < UG; ++q)
+#pragma unroll
+                    for (int e = 0; e < IPL; ++e)
+                        if (src[q][e] >= 0) {
+                            const int va = (e * 32 + lane) % RV;
+                            const int j = (g0 + q * NWALL) * GR + (e * 32 + lane) / RV;
+                            uint16_t* dp = va >= G::VPR ? dstV : dstK;
+                            st_stream(reinterpret_cast<uint4*>(dp + (long long)j * G::D) + (va % G::VPR), buf[q][e]);
+                        }
             }
         }
     }

@@ -22,8 +22,10 @@ from paper_2504_04704_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-SCORE_ABS_TOL = 1e-4     # binding tolerance on scores
-SCORE_REL_TOL = 2e-5     # tight: |gpu - oracle| <= SCORE_REL_TOL * (2 / L)
+import parity_util as pu
+
+SCORE_ABS_TOL = pu.SCORE_ABS_TOL     # binding tolerance on scores: 1e-4 absolute
+SCORE_REL_TOL = pu.SCORE_REL_TOL     # tight: |gpu - oracle| <= 1e-5 * (2 / L)
 
 
 @pytest.fixture(scope="module")
@@ -47,39 +49,7 @@ def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, vari
     if n_c == 0:
         np.testing.assert_array_equal(idx, ref["idx"])
         return {"mismatch_partitions": 0, "max_abs": 0.0, "max_rel": 0.0}
-    # sink and window
-    np.testing.assert_array_equal(idx[..., :sink], ref["idx"][..., :sink])
-    np.testing.assert_array_equal(idx[..., sink + n_c * k:], ref["idx"][..., sink + n_c * k:])
-    # scores
-    gs = out["scores"].astype(np.float64)
-    err = np.abs(gs - ref["scores"])
-    max_abs = float(err.max())
-    max_rel = float(err.max() * L / 2.0)
-    assert max_abs <= SCORE_ABS_TOL, f"score error {max_abs}"
-    assert max_rel <= SCORE_REL_TOL, f"score error relative to 2/L: {max_rel}"
-    # the GPU's selection is the exact top-k of its own fp32 scores
-    s32 = out["scores"]
-    order = np.argsort(-s32, axis=-1, kind="stable")[..., :k]
-    own = np.sort(order, axis=-1) + (sink + np.arange(n_c) * L)[None, None, :, None]
-    got = idx[..., sink:sink + n_c * k].reshape(B, H, n_c, k)
-    np.testing.assert_array_equal(got, own)
-    # index sets against the oracle
-    want = ref["idx"][..., sink:sink + n_c * k].reshape(B, H, n_c, k)
-    bad = np.argwhere((got != want).any(-1))
-    loose_unexplained = tight_unexplained = 0
-    for b, h, p in bad:
-        sc = ref["scores"][b, h, p]
-        srt = np.sort(sc)[::-1]
-        gap = srt[k - 1] - srt[k] if k < L else np.inf
-        if gap >= SCORE_ABS_TOL:
-            loose_unexplained += 1
-        eps = err[b, h, p].max()
-        diff = np.setxor1d(got[b, h, p], want[b, h, p]) - (sink + p * L)
-        if np.any(np.abs(sc[diff] - srt[k - 1]) > 2 * eps):
-            tight_unexplained += 1
-    assert loose_unexplained == 0
-    assert tight_unexplained == 0
-    res = {"mismatch_partitions": int(len(bad)), "partitions": int(B * H * n_c), "max_abs": max_abs, "max_rel": max_rel}
+    res = pu.compare_with_oracle(ref, out, sink, L, k, abs_tol=SCORE_ABS_TOL, rel_tol=SCORE_REL_TOL)
     if stats is not None:
         stats.update(res)
     return res
@@ -250,6 +220,35 @@ def test_indices_only_and_rows_only(binding, oracle, warps):
     only_rows = plan.compress_prefill(K, V, ws, want_idx=False)
     assert torch.equal(full["idx"], only_idx["idx"])
     assert torch.equal(full["K_out"], only_rows["K_out"]) and torch.equal(full["V_out"], only_rows["V_out"])
+    assert plan.read_status(ws)[0] == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("D", [64, 96, 128, 256])
+def test_rows_only_warp_specialised_every_head_dim(binding, oracle, D, dtype):
+    """Rows without indices on the warp-specialised kernel: the kept positions are parked in the
+    output rows themselves and read back by the copy warp and the final gather, whose lane-to-row
+    mapping depends on head_dim.  Many slots per CTA, outputs poisoned before every run; the rows
+    must equal those of the run that also returns indices, which is checked against the oracle."""
+    B, H, sink, L, k = 8, 5, 16, 256, 64
+    S = sink + 21 * L + 77                     # 40 units x 21 slots: five or six slots per CTA
+    K, V = synth.make_kv(B, H, S, D, seed=300 + D, device="cuda:0", dtype=dtype)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0, dtype=dtype)
+    info = plan.launch_info(S)
+    assert info["kernel"] == "lagkv_ws_kernel" and info["grid"] * 4 < B * H * 21
+    ws = plan.new_workspace()
+    full = plan.compress_prefill(K, V, ws, want_scores=True)
+    assert plan.read_status(ws)[0] == 0
+    host = {"L_R": full["L_R"], "idx": full["idx"].cpu().numpy(), "K_out": synth.to_bits(full["K_out"]),
+            "V_out": synth.to_bits(full["V_out"]), "scores": full["scores"].cpu().numpy()}
+    check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host,
+                         storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
+    L_R = full["L_R"]
+    for run in range(6):
+        out = {"K_out": torch.full((B, H, L_R, D), -3.0, dtype=dtype, device="cuda:0"),
+               "V_out": torch.full((B, H, L_R, D), -3.0, dtype=dtype, device="cuda:0")}
+        res = plan.compress_prefill(K, V, ws, out=out, want_idx=False)
+        assert torch.equal(res["K_out"], full["K_out"]) and torch.equal(res["V_out"], full["V_out"]), f"run {run}"
     assert plan.read_status(ws)[0] == 0
 
 

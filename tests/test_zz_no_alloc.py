@@ -7,7 +7,8 @@ under a policy that forbids ``cudaMalloc`` after start-up.  They cannot supply t
 this entry point uses it.  The checks here: through the C ABI, on two calls in a row (the
 array is shared and keeps the previous call's contents), the result is identical to the
 workspace-taking entry point's -- caches, lengths and kept positions bit for bit, which is
-the bar the other append tests use -- and a request beyond the array's size is refused.
+the bar the other append tests use -- and to the float64 oracle's replay of the same append;
+a request beyond the array's size is refused.
 
 This file sorts last on purpose: a run that stops at the first failure has then already
 gone through every other test.
@@ -34,8 +35,8 @@ def _case(seed, B, H, D, S_cap, seq, stat):
             torch.tensor(stat, dtype=torch.int32, device="cuda:0"))
 
 
-def _run_both(binding, plan, ws, case, max_chunks, give_idx):
-    """Same inputs through the workspace entry point and through the no-allocation one."""
+def _run_both(binding, oracle, plan, ws, case, max_chunks, give_idx):
+    """Same inputs through the workspace entry point, the no-allocation one and the oracle."""
     B, H, k = plan.cfg.B, plan.cfg.H_kv, plan.k
     K, V, seq, stat = case
     Ka, Va, seqa, stata = K.clone(), V.clone(), seq.clone(), stat.clone()
@@ -53,20 +54,31 @@ def _run_both(binding, plan, ws, case, max_chunks, give_idx):
     if give_idx:
         assert torch.equal(idxa, idxb)
     assert not torch.equal(seqb, seq), "the case must trigger at least one compression"
+    # the oracle's replay of the same append: lengths, rows up to the new length, kept positions
+    Kr, Vr, seqr, statr, kept = oracle.compress_append(synth.to_bits(K), synth.to_bits(V), seq.cpu().numpy(),
+                                                       stat.cpu().numpy(), plan.cfg.lag, k)
+    assert seqb.tolist() == seqr.tolist() and statb.tolist() == statr.tolist()
+    Kg, Vg = synth.to_bits(Kb), synth.to_bits(Vb)
+    for b in range(B):
+        m = int(seqr[b])
+        np.testing.assert_array_equal(Kg[b, :, :m], Kr[b, :, :m])
+        np.testing.assert_array_equal(Vg[b, :, :m], Vr[b, :, :m])
+        if give_idx and kept[b].shape[1]:
+            np.testing.assert_array_equal(idxb[b, :, :kept[b].shape[1]].cpu().numpy(), kept[b])
     return status.tolist()
 
 
-def test_noalloc_matches_workspace_entry_point_twice_in_a_row(binding):
+def test_noalloc_matches_workspace_entry_point_twice_in_a_row(binding, oracle):
     B, H, D, sink, L, k = 3, 2, 128, 8, 64, 16
     plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
     ws = plan.new_workspace(3)
     # first call: kept positions parked in the library's scratch (no idx_out), several chunks
     c1 = _case(101, B, H, D, 600, [sink + 4 * L + 3, sink + 2 * L, sink + 2 * L - 1], [sink, sink, sink])
-    st1 = _run_both(binding, plan, ws, c1, 3, give_idx=False)
+    st1 = _run_both(binding, oracle, plan, ws, c1, 3, give_idx=False)
     assert st1[0] == 0
     # second call right behind it, other data and lengths: nothing of the first call may leak in
     c2 = _case(202, B, H, D, 600, [sink + 3 * k + 2 * L + 9, sink + 3 * L + 1, sink + L], [sink + 3 * k, sink, sink])
-    st2 = _run_both(binding, plan, ws, c2, 3, give_idx=True)
+    st2 = _run_both(binding, oracle, plan, ws, c2, 3, give_idx=True)
     assert st2[0] == 0
     # third: a device-side error code must show up in status_out and must not stick afterwards
     c3 = _case(303, B, H, D, 600, [sink + 5 * L, sink + 2 * L, sink + 2 * L], [sink, sink, sink])   # needs 4 chunks
@@ -74,7 +86,11 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(binding):
     status = torch.zeros(4, dtype=torch.int32, device="cuda:0")
     plan.compress_append_noalloc(K, V, seq, stat, max_new_chunks=3, status_out=status)
     assert status.tolist()[0] == binding.LAGKV_ECAPACITY
-    st4 = _run_both(binding, plan, ws, c1, 3, give_idx=False)
+    # without status_out the code waits in the built-in scratch until it is read (or the next call clears it)
+    plan.compress_append_noalloc(K, V, seq, stat, max_new_chunks=3)
+    assert plan.read_status(None)[0] == binding.LAGKV_ECAPACITY
+    assert plan.read_status(None)[0] == 0
+    st4 = _run_both(binding, oracle, plan, ws, c1, 3, give_idx=False)
     assert st4[0] == 0
 
 
@@ -90,6 +106,16 @@ def test_noalloc_refuses_what_does_not_fit(binding):
     with pytest.raises(binding.LagKVError) as e:
         plan.compress_append_noalloc(K, V, seq, stat, max_new_chunks=2)
     assert e.value.code == binding.LAGKV_ENOALLOC_LIMIT
+    # an argument the host refuses must not clear what the previous call left in the scratch
+    small = binding.Plan(2, 1, D, 4, 8, keep_k=8, device=0)
+    k2, v2 = torch.zeros((2, 1, 64, D), dtype=torch.bfloat16, device="cuda:0"), torch.zeros((2, 1, 64, D), dtype=torch.bfloat16, device="cuda:0")
+    s2 = torch.tensor([4 + 5 * 8, 4], dtype=torch.int32, device="cuda:0")
+    t2 = torch.tensor([4, 4], dtype=torch.int32, device="cuda:0")
+    small.compress_append_noalloc(k2, v2, s2, t2, max_new_chunks=1)             # needs 4 chunks: ECAPACITY on the device
+    with pytest.raises(binding.LagKVError) as e2:
+        small.compress_append_noalloc(k2, k2, s2, t2, max_new_chunks=1)         # K and V alias: refused on the host
+    assert e2.value.code == binding.LAGKV_EINVAL
+    assert small.read_status(None)[0] == binding.LAGKV_ECAPACITY
     assert "scratch" in binding.status_string(binding.LAGKV_ENOALLOC_LIMIT)
     assert seq.tolist() == [8] * B
     # with idx_out supplied only the status block is needed, so the same shape is accepted
