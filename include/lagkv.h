@@ -292,6 +292,16 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]);
  * fit shared memory.
  */
 #define LAGKV_TUNE_PAIRS 100
+/*
+ * warps = LAGKV_TUNE_APPEND_CLUSTER (4 warps per CTA) or LAGKV_TUNE_APPEND_CLUSTER8 (8 warps,
+ * head_dim 128 only) shapes the kernel of one-partition appends (lagkv_compress_append with
+ * max_new_chunks == 1, LagKV scoring) instead: tile_rows = row splits per tensor (1, 2 or 4: a
+ * cluster of 2, 4 or 8 CTAs per (b, h) unit), stages = ring stages (2..4), ctas_per_sm = CTAs
+ * per SM to leave room for (1..4; fewer resident rows of the window when they do not all fit,
+ * which only a split of 1 allows).  The prefill shape is left alone.
+ */
+#define LAGKV_TUNE_APPEND_CLUSTER 101
+#define LAGKV_TUNE_APPEND_CLUSTER8 102
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages,
                     int32_t ctas_per_sm);
 

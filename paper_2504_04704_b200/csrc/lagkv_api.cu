@@ -37,6 +37,8 @@ struct KernelTable {
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = pair_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = append_pair_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
     }
 };
 const KernelTable& table() {
@@ -76,7 +78,11 @@ struct lagkv_plan_s {
     Shape pre;        // kernel used by lagkv_compress_prefill
     Shape pair;       // pair kernel, preferred for short partitions with enough of them (kidx < 0: none)
     bool tuned;       // lagkv_plan_tune() fixed the prefill kernel: no switching by size
-    Shape app;        // kernel used by lagkv_compress_append (always the uniform kernel)
+    Shape app;        // uniform kernel of lagkv_compress_append (any number of partitions per call)
+    Shape app_pair;   // one-partition appends: a cluster of two CTAs per unit (kidx < 0: none)
+    int app_pair_res_tiles;  // tiles of the window a CTA keeps in shared memory
+    int app_pair_splits;     // row splits per tensor: the cluster has twice as many CTAs
+    bool app_tuned;   // lagkv_plan_tune() fixed the uniform append shape: no pair kernel
     // lagkv_compress_prefill_host(): three streams and the events between them, made on first use
     std::mutex host_mu;
     bool host_ready = false;
@@ -123,6 +129,17 @@ int keep_count(double r, int L) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The dynamic shared memory limit belongs to the function, not to the plan: only ever raise it, so
+// that shapes of the same kernel with larger needs (this plan's or another's) keep launching.
+bool raise_smem_limit(const void* fn, size_t smem) {
+    static std::mutex limit_mu;  // read-then-raise must not interleave between threads
+    std::lock_guard<std::mutex> lock(limit_mu);
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return false;
+    return size_t(attr.maxDynamicSharedSizeBytes) >= smem ||
+           cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) == cudaSuccess;
+}
+
 // Try one launch shape (NW = warps per CTA, 12 = the warp-specialised kernel).
 int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Shape* out) {
     const int kidx = find_kernel(pl->cfg.D, NW, TR, pl->cfg.variant, pl->cfg.dtype);
@@ -132,22 +149,43 @@ int make_shape(const lagkv_plan_s* pl, int NW, int TR, int stages, int ctas, Sha
     const size_t smem = kKernels[kidx].smem(stages, pl->cfg.lag);
     if (smem > size_t(pl->max_smem_optin)) return LAGKV_EUNSUPPORTED;
     if ((smem + 1024) * size_t(ctas) > size_t(kSmemPerSm)) return LAGKV_EUNSUPPORTED;
-    if (pl->cfg.device >= 0) {
-        // the limit belongs to the function, not to the plan: only ever raise it, so that shapes of
-        // the same kernel with deeper rings (this plan's or another's) keep launching
-        const void* fn = reinterpret_cast<const void*>(kKernels[kidx].fn);
-        static std::mutex limit_mu;  // read-then-raise must not interleave between threads
-        std::lock_guard<std::mutex> lock(limit_mu);
-        cudaFuncAttributes attr;
-        if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return LAGKV_ECUDA;
-        if (size_t(attr.maxDynamicSharedSizeBytes) < smem &&
-            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-            return LAGKV_ECUDA;
-    }
+    if (pl->cfg.device >= 0 && !raise_smem_limit(reinterpret_cast<const void*>(kKernels[kidx].fn), smem))
+        return LAGKV_ECUDA;
     out->kidx = kidx;
     out->stages = stages;
     out->ctas_per_sm = ctas;
     out->smem = smem;
+    return LAGKV_OK;
+}
+
+// Shape of the one-partition append kernel: `code` = LAGKV_TUNE_APPEND_CLUSTER / _CLUSTER8, `splits`
+// row splits per tensor, room for `ctas` CTAs per SM.  `full` demands that the whole window stays
+// resident (mandatory with more than one split).
+int make_append_cluster(lagkv_plan_s* pl, int code, int splits, int stages, int ctas, bool full) {
+    if (splits != 1 && splits != 2 && splits != 4) return LAGKV_EUNSUPPORTED;
+    if (stages < 2 || stages > 4 || ctas < 1 || ctas > 4) return LAGKV_EUNSUPPORTED;
+    const int kidx = find_kernel(pl->cfg.D, code, kAppendPairTileRows, LAGKV_VARIANT_LAGKV, pl->cfg.dtype);
+    if (kidx < 0 || pl->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
+    const int L = pl->cfg.lag;
+    const size_t rowb = size_t(pl->cfg.D) * 2, per_tile = size_t(kAppendPairTileRows) * rowb + 8;
+    const size_t fixed = kKernels[kidx].smem(stages, L);
+    size_t budget = size_t(kSmemPerSm) / size_t(ctas) - 1024;
+    if (budget > size_t(pl->max_smem_optin)) budget = size_t(pl->max_smem_optin);
+    if (fixed > budget) return LAGKV_EUNSUPPORTED;
+    const int ntiles = (L + kAppendPairTileRows - 1) / kAppendPairTileRows;
+    const int nloc = (ntiles + splits - 1) / splits;  // tiles of the largest share
+    long long fit = (long long)((budget - fixed) / per_tile);
+    const int res_tiles = int(fit < nloc ? fit : nloc);
+    if ((full || splits > 1) && res_tiles < nloc) return LAGKV_EUNSUPPORTED;
+    // with row splits a CTA gathers its share of the kept rows into the rings in one go
+    const size_t ring = size_t(kKernels[kidx].threads / 32) * stages * kAppendPairTileRows * rowb;
+    if (splits > 1 && size_t((pl->k + splits - 1) / splits) * rowb > ring) return LAGKV_EUNSUPPORTED;
+    const size_t smem = fixed + size_t(res_tiles) * per_tile;
+    if (pl->cfg.device >= 0 && !raise_smem_limit(reinterpret_cast<const void*>(kKernels[kidx].fn), smem))
+        return LAGKV_ECUDA;
+    pl->app_pair = Shape{kidx, stages, ctas, smem};
+    pl->app_pair_res_tiles = res_tiles;
+    pl->app_pair_splits = splits;
     return LAGKV_OK;
 }
 
@@ -193,6 +231,22 @@ int choose_shape(lagkv_plan_s* pl) {
     }
     pl->pair.kidx = -1;
     pl->tuned = false;
+    pl->app_tuned = false;
+    pl->app_pair.kidx = -1;
+    // one-partition appends (decode): the smallest cluster whose CTAs keep the whole window
+    // resident with two CTAs to an SM, else the pair of CTAs with as much of it as fits
+    if (pl->cfg.variant == LAGKV_VARIANT_LAGKV) {
+        bool found = false;
+        for (int splits = 1; splits <= kAppendMaxSplits && !found; splits *= 2) {
+            const int rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, splits, 2, 2, true);
+            if (rc2 == LAGKV_ECUDA) return rc2;
+            found = rc2 == LAGKV_OK;
+        }
+        if (!found) {
+            const int rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, 1, 2, 1, false);
+            if (rc2 == LAGKV_ECUDA) return rc2;
+        }
+    }
     if (L >= 256) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
         Shape sh;
@@ -283,7 +337,7 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
     if (cfg->dtype != LAGKV_DTYPE_BF16 && cfg->dtype != LAGKV_DTYPE_FP16) return LAGKV_EINVAL;
     if (cfg->D != 64 && cfg->D != 96 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
-    if ((long long)cfg->B * cfg->H_kv > (1ll << 30) || cfg->H_kv >= kSeqFailed) return LAGKV_EINVAL;
+    if ((long long)cfg->B * cfg->H_kv > (1ll << 30) || 8 * (long long)cfg->H_kv >= kSeqFailed) return LAGKV_EINVAL;
 
     lagkv_plan_s* pl = new (std::nothrow) lagkv_plan_s();
     if (pl == nullptr) return LAGKV_EINVAL;
@@ -620,9 +674,32 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     P.max_chunks = max_new_chunks;
     P.stages = plan->app.stages;
 
-    const KernelEntry& ke = kKernels[plan->app.kidx];
     const long long U = (long long)c.B * c.H_kv;
     void* args[] = {&P};
+    if (max_new_chunks == 1 && plan->app_pair.kidx >= 0 && !plan->app_tuned) {
+        // decode: at most one partition per sequence and call -> a cluster of CTAs per unit
+        const KernelEntry& kp = kKernels[plan->app_pair.kidx];
+        P.idx_out = idx_out;
+        P.stages = plan->app_pair.stages;
+        P.res_tiles = plan->app_pair_res_tiles;
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof cfg);
+        const unsigned cs = 2u * unsigned(plan->app_pair_splits);
+        cfg.gridDim = dim3((unsigned)(cs * U));
+        cfg.blockDim = dim3(kp.threads);
+        cfg.dynamicSmemBytes = plan->app_pair.smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = cs;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(kp.fn), args) != cudaSuccess) return LAGKV_ECUDA;
+        return check_launch();
+    }
+    const KernelEntry& ke = kKernels[plan->app.kidx];
     if (cudaLaunchKernel(reinterpret_cast<const void*>(ke.fn), dim3((unsigned)U), dim3(ke.NW * 32), args,
                          plan->app.smem, stream) != cudaSuccess)
         return LAGKV_ECUDA;
@@ -703,6 +780,13 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]) {
 int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t stages, int32_t ctas_per_sm) {
     if (plan == nullptr) return LAGKV_EINVAL;
     DeviceGuard guard(plan->cfg.device);
+    if (warps == LAGKV_TUNE_APPEND_CLUSTER || warps == LAGKV_TUNE_APPEND_CLUSTER8) {
+        const int splits = tile_rows ? tile_rows : (plan->app_pair.kidx >= 0 ? plan->app_pair_splits : 1);
+        const int st = stages ? stages : 2, ct = ctas_per_sm ? ctas_per_sm : 1;
+        const int rc = make_append_cluster(plan, warps, splits, st, ct, false);
+        if (rc == LAGKV_OK) plan->app_tuned = false;
+        return rc;
+    }
     const KernelEntry& cur = kKernels[plan->pre.kidx];
     Shape sh;
     const int rc = make_shape(plan, warps ? warps : cur.NW, tile_rows ? tile_rows : cur.TR,
@@ -711,7 +795,10 @@ int lagkv_plan_tune(lagkv_plan_t plan, int32_t warps, int32_t tile_rows, int32_t
     if (rc != LAGKV_OK) return rc;
     plan->pre = sh;
     plan->tuned = true;
-    if (!kKernels[sh.kidx].ws) plan->app = sh;
+    if (!kKernels[sh.kidx].ws) {
+        plan->app = sh;
+        plan->app_tuned = true;
+    }
     return LAGKV_OK;
 }
 

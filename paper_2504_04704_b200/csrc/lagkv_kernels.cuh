@@ -52,6 +52,7 @@ struct Params {
     int max_chunks;               // append
     int stages;                   // ring depth per warp
     int sel_emit;                 // warp-specialised kernel: select warps move the kept rows of odd slots
+    int res_tiles;                // append pair kernel: tiles of the window that stay in shared memory
 };
 
 // ------------------------------------------------------------------------------ PTX helpers
@@ -297,8 +298,9 @@ __device__ __forceinline__ void transposed_reduce(float (&v)[NV], int cg) {
 
 // ---------------------------------------------------------------------------- tile math
 // One staged tile of one tensor: rows [0, nrows) valid.  Updates the packed per-channel
-// min / max; when SCORE, also writes sigma (Std. of Eq. 10) for every valid row.
-template <class G, bool SCORE, bool FULL>
+// min / max (unless STATS is off: a partition nobody takes statistics from); when SCORE, also
+// writes sigma (Std. of Eq. 10) for every valid row.
+template <class G, bool SCORE, bool FULL, bool STATS = true>
 __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int nrows,
                                              const f32x2 (&a2)[G::NWORD], const f32x2 (&b2)[G::NWORD],
                                              uint32_t (&mn)[G::NWORD], uint32_t (&mx)[G::NWORD],
@@ -318,7 +320,7 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int j = v * 4 + c;
-                if (valid) {
+                if (STATS && valid) {
                     mn[j] = G::E::min2(mn[j], w[c]);
                     mx[j] = G::E::max2(mx[j], w[c]);
                 }

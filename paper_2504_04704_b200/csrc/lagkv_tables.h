@@ -6,6 +6,7 @@
 #include "lagkv_kernels.cuh"
 #include "lagkv_ws_kernel.cuh"
 #include "lagkv_pair_kernel.cuh"
+#include "lagkv_append_pair_kernel.cuh"
 
 namespace lagkv {
 
@@ -31,6 +32,11 @@ int ws_kernels(const KernelEntry** table);            // lagkv_ws_kernel: warp-s
 int ws_dims_kernels(const KernelEntry** table);
 int ws_dims_fp16_kernels(const KernelEntry** table);
 int pair_kernels(const KernelEntry** table);          // lagkv_pair_kernel: prefill, short partitions
+// lagkv_append_pair_kernel: one-partition appends on a cluster of 2, 4 or 8 CTAs per unit.  NW
+// holds LAGKV_TUNE_APPEND_CLUSTER (4 warps per CTA) or LAGKV_TUNE_APPEND_CLUSTER8 (8 warps);
+// smem() gives the size without resident tiles (TILE_BYTES + 8 each).
+int append_pair_kernels(const KernelEntry** table);
+constexpr int kAppendPairTileRows = 16;
 
 // ---- table entries: (head_dim, vectors per lane, warps, tile rows, variant, element format)
 #define LAGKV_ENTRY2(D, V, NW, TR, VAR, DT) \

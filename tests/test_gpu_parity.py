@@ -538,6 +538,82 @@ def test_append_single_chunk_ragged_batch(binding, oracle):
         np.testing.assert_array_equal(r["K"][b, :, seq[b]:], r["K0"][b, :, seq[b]:])
 
 
+CLUSTER = 101      # LAGKV_TUNE_APPEND_CLUSTER: 4 warps per CTA
+CLUSTER8 = 102     # LAGKV_TUNE_APPEND_CLUSTER8: 8 warps per CTA (head_dim 128)
+
+
+@pytest.mark.parametrize("code,splits,stages,ctas,D,L,k,dtype", [
+    (CLUSTER, 1, 2, 2, 128, 64, 16, torch.bfloat16), (CLUSTER, 2, 2, 2, 128, 64, 16, torch.bfloat16),
+    (CLUSTER, 4, 2, 2, 128, 72, 9, torch.bfloat16), (CLUSTER, 2, 3, 1, 128, 512, 128, torch.bfloat16),
+    (CLUSTER, 4, 2, 3, 128, 512, 128, torch.float16), (CLUSTER, 1, 2, 1, 128, 512, 128, torch.bfloat16),
+    (CLUSTER, 1, 2, 1, 128, 2048, 700, torch.bfloat16),     # pair of CTAs, window only partly resident
+    (CLUSTER, 1, 2, 2, 128, 512, 128, torch.bfloat16),      # the same at L = 512 (two CTAs to an SM)
+    (CLUSTER8, 1, 2, 1, 128, 512, 128, torch.bfloat16), (CLUSTER8, 2, 2, 1, 128, 1024, 256, torch.float16),
+    (CLUSTER, 2, 2, 2, 64, 256, 64, torch.bfloat16), (CLUSTER, 4, 2, 1, 96, 200, 50, torch.float16),
+    (CLUSTER, 2, 2, 1, 256, 256, 32, torch.bfloat16), (CLUSTER, 1, 2, 1, 256, 1024, 1, torch.float16),
+    (CLUSTER, 2, 2, 2, 128, 37, 37, torch.bfloat16),        # k = L: nothing moves, only the lengths change
+    (CLUSTER, 4, 2, 2, 128, 20, 3, torch.bfloat16),         # fewer tiles than row splits
+])
+def test_append_cluster_shapes(binding, oracle, code, splits, stages, ctas, D, L, k, dtype):
+    """One-partition appends on every cluster shape: a ragged batch (some sequences trigger with and
+    without a remainder, one skips, one asks for two partitions and is refused) against the
+    oracle's replay, kept positions included."""
+    sink = 8
+    stat = [sink, sink + 3 * k, sink + k, sink, sink + 2 * k]
+    seq = [stat[0] + 2 * L, stat[1] + 2 * L + L - 1, stat[2] + 2 * L + 5, stat[3] + 2 * L - 1, stat[4] + 3 * L]
+    S_cap = max(seq) + 7
+    B, H = 5, 3
+    r = append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, 1, seed=L + k + splits, dtype=dtype,
+                    tune=dict(warps=code, tile_rows=splits, stages=stages, ctas_per_sm=ctas))
+    assert r["status"][0] == binding.LAGKV_ECAPACITY          # the last sequence needs two partitions
+    for b in range(4):
+        n = int(r["seq_r"][b])
+        assert r["seq"][b] == r["seq_r"][b] and r["stat"][b] == r["stat_r"][b]
+        np.testing.assert_array_equal(r["K"][b, :, :n], r["Kr"][b, :, :n])
+        np.testing.assert_array_equal(r["V"][b, :, :n], r["Vr"][b, :, :n])
+        np.testing.assert_array_equal(r["K"][b, :, seq[b]:], r["K0"][b, :, seq[b]:])     # nothing beyond the old length
+        if r["kept"][b].shape[1]:
+            np.testing.assert_array_equal(r["idx"][b, :, :k], r["kept"][b])
+    assert r["seq"][3] == seq[3] and r["seq"][4] == seq[4] and r["stat"][4] == stat[4]
+    np.testing.assert_array_equal(r["K"][3:], r["K0"][3:])
+    np.testing.assert_array_equal(r["V"][3:], r["V0"][3:])
+
+
+@pytest.mark.parametrize("splits,layout", [(1, "padded"), (2, "bshd"), (4, "padded")])
+def test_append_cluster_strided(binding, oracle, splits, layout):
+    """Cluster appends on caches whose rows are not contiguous: row-by-row copies everywhere."""
+    B, H, D, sink, L, k = 3, 2, 128, 4, 96, 24
+    stat = [sink, sink + k, sink]
+    seq = [stat[0] + 2 * L + 11, stat[1] + 2 * L, stat[2] + L]
+    S_cap = max(seq) + 3
+    K, V = synth.make_kv(B, H, S_cap, D, seed=5 + splits, device="cuda:0")
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    if layout == "bshd":
+        Kd = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        Vd = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        strides = (S_cap * H * D, D, H * D)
+    else:
+        Kp = torch.zeros((B, H, S_cap, D + 8), dtype=torch.bfloat16, device="cuda:0")
+        Vp = torch.zeros_like(Kp)
+        Kp[..., :D], Vp[..., :D] = K, V
+        Kd, Vd = Kp[..., :D], Vp[..., :D]
+        strides = (H * S_cap * (D + 8), S_cap * (D + 8), D + 8)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, strides=strides, device=0)
+    plan.tune(warps=CLUSTER, tile_rows=splits, stages=2, ctas_per_sm=2)
+    ws = plan.new_workspace(1)
+    seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
+    stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
+    plan.compress_append(Kd, Vd, seq_d, stat_d, ws, max_new_chunks=1)
+    assert plan.read_status(ws)[0] == 0
+    Kr, Vr, seq_r, stat_r, _ = oracle.compress_append(Kb, Vb, np.array(seq), np.array(stat), L, k)
+    assert seq_d.tolist() == seq_r.tolist() and stat_d.tolist() == stat_r.tolist()
+    Kg, Vg = synth.to_bits(Kd.contiguous()), synth.to_bits(Vd.contiguous())
+    for b in range(B):
+        n = int(seq_r[b])
+        np.testing.assert_array_equal(Kg[b, :, :n], Kr[b, :, :n])
+        np.testing.assert_array_equal(Vg[b, :, :n], Vr[b, :, :n])
+
+
 @pytest.mark.parametrize("L,k,chunks", [(64, 16, 4), (96, 96, 2), (256, 1, 3), (512, 128, 2)])
 def test_append_multi_chunk(binding, oracle, L, k, chunks):
     sink = 8
