@@ -207,6 +207,46 @@ int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64
                           size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Paged caches (block tables).  The method itself (Section 2.2) only speaks of a cache of n
+ * rows per head; serving engines store that cache as fixed-size pages drawn from a pool, with a
+ * table per sequence saying which page holds which rows.  K_pool / V_pool are DEVICE pointers to
+ * pools addressed as
+ *     pool + block_table[b*max_blocks + s/page_size]*stride_page + h*stride_h + (s%page_size)*stride_s + d
+ * (the same table and strides for K and V).  A stride given as 0 means dense
+ * [num_pages, H_kv, page_size, D].  With layers folded into B, sequence b's table row simply
+ * names pages of its own layer.  The plan's own strides must be 0.
+ */
+typedef struct {
+    const int32_t *block_table; /* DEVICE int32 [B, max_blocks], 4-byte aligned               */
+    int32_t max_blocks;         /* entries per sequence; max_blocks*page_size >= rows addressed */
+    int32_t page_size;          /* rows per page: a power of two, >= 16                        */
+    int64_t stride_page;        /* elements between pages          (0 = H_kv*stride_h)         */
+    int64_t stride_h;           /* elements between heads in a page (0 = page_size*stride_s)   */
+    int64_t stride_s;           /* elements between rows in a page  (0 = D); multiples of 8    */
+} lagkv_paged_layout;
+
+/*
+ * lagkv_compress_prefill() reading a paged cache (same pass, Section 2.2, Eq. 7-12): every
+ * sequence has S_in rows; the outputs are contiguous as there.  Runs on the kernel family that
+ * looks rows up page by page (a tile that straddles a page boundary is fetched in two copies).
+ */
+int lagkv_compress_prefill_paged(lagkv_plan_t plan, const void *K_pool, const void *V_pool,
+                                 const lagkv_paged_layout *layout, int64_t S_in, void *K_out, void *V_out,
+                                 int32_t *idx_out, float *scores_out, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream);
+
+/*
+ * lagkv_compress_append() in place on a paged cache (Section 2.2, bullets 2-4; Fig. 1): kept rows
+ * and the window are moved down inside the sequence's own pages, seq_len / static_len are
+ * updated as there.  A sequence may hold at most max_blocks*page_size rows.  Pages that lie wholly
+ * behind the new seq_len[b] hold no valid rows any more; giving them back to the pool is the
+ * caller's business (the table is not modified).
+ */
+int lagkv_compress_append_paged(lagkv_plan_t plan, void *K_pool, void *V_pool, const lagkv_paged_layout *layout,
+                                int32_t *seq_len, int32_t *static_len, int32_t max_new_chunks, int32_t *idx_out,
+                                float *scores_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * lagkv_compress_append() for callers that have no device memory to give as a workspace.
  * (The paper has no counterpart: this is a property of the library, not of the method.)
  *

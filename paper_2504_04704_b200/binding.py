@@ -29,7 +29,8 @@ EXPORTS = (
     "lagkv_plan", "lagkv_plan_destroy", "lagkv_keep_count", "lagkv_compressed_len",
     "lagkv_keep_for_target", "lagkv_lengths_after", "lagkv_workspace_bytes", "lagkv_workspace_init",
     "lagkv_compress_prefill", "lagkv_compress_prefill_host", "lagkv_host_staging_bytes",
-    "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_gather",
+    "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_compress_prefill_paged",
+    "lagkv_compress_append_paged", "lagkv_gather",
     "lagkv_read_status",
     "lagkv_launch_info", "lagkv_plan_tune", "lagkv_selftest_bounded_wait", "lagkv_status_string", "lagkv_version",
 )
@@ -49,6 +50,13 @@ class lagkv_config(ctypes.Structure):
         ("keep_k", ctypes.c_int32), ("std_ddof", ctypes.c_int32), ("variant", ctypes.c_int32),
         ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_s", ctypes.c_int64),
         ("device", ctypes.c_int32), ("dtype", ctypes.c_int32),
+    ]
+
+
+class lagkv_paged_layout(ctypes.Structure):
+    _fields_ = [
+        ("block_table", ctypes.c_void_p), ("max_blocks", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("stride_page", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_s", ctypes.c_int64),
     ]
 
 
@@ -92,6 +100,12 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_compress_append.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.lagkv_compress_append_noalloc.restype = ctypes.c_int
     lib.lagkv_compress_append_noalloc.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
+    lib.lagkv_compress_prefill_paged.restype = ctypes.c_int
+    lib.lagkv_compress_prefill_paged.argtypes = [vp, vp, vp, ctypes.POINTER(lagkv_paged_layout), i64, vp, vp, vp, vp, vp,
+                                                 sz, vp]
+    lib.lagkv_compress_append_paged.restype = ctypes.c_int
+    lib.lagkv_compress_append_paged.argtypes = [vp, vp, vp, ctypes.POINTER(lagkv_paged_layout), vp, vp, i32, vp, vp, vp,
+                                                sz, vp]
     lib.lagkv_gather.restype = ctypes.c_int
     lib.lagkv_gather.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
     lib.lagkv_read_status.restype = ctypes.c_int
@@ -279,6 +293,52 @@ class Plan:
             self.handle, _ptr(K_cache), _ptr(V_cache), int(K_cache.shape[2]), _ptr(seq_len), _ptr(static_len),
             int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(status_out), _stream(self._dev()))
         _check(rc, "lagkv_compress_append_noalloc")
+
+    def _paged(self, K_pool, block_table, strides):
+        """``lagkv_paged_layout`` of a pool ``[num_pages, H, page_size, D]`` (or ``strides`` = (page, head,
+        row) in elements for another arrangement) and an int32 CUDA table ``[B, max_blocks]``."""
+        if block_table.dtype != torch.int32 or not block_table.is_cuda or not block_table.is_contiguous() or \
+                block_table.dim() != 2 or block_table.shape[0] != self.cfg.B:
+            raise TypeError("block_table must be a contiguous int32 CUDA tensor [B, max_blocks]")
+        sp, sh, ss = strides[:3] if strides is not None else (0, 0, 0)
+        page_size = int(K_pool.shape[2]) if strides is None else int(strides[3])
+        return lagkv_paged_layout(block_table.data_ptr(), int(block_table.shape[1]), page_size, int(sp), int(sh), int(ss))
+
+    def compress_prefill_paged(self, K_pool, V_pool, block_table, S_in, workspace, want_scores=False, strides=None):
+        """``lagkv_compress_prefill_paged``: pools ``[num_pages, H, page_size, D]`` (``strides`` =
+        (page, head, row, page_size) for another arrangement), table ``[B, max_blocks]``; the
+        outputs are contiguous as for ``compress_prefill``."""
+        self._check_cache(K_pool, "K_pool")
+        self._check_cache(V_pool, "V_pool")
+        lay = self._paged(K_pool, block_table, strides)
+        c, dev = self.cfg, self._dev()
+        L_R = self.compressed_len(S_in)
+        rest = S_in - c.sink
+        n_c = rest // c.lag - 1 if rest >= 2 * c.lag else 0
+        out = {"K_out": torch.empty((c.B, c.H_kv, L_R, c.D), dtype=self.dtype, device=dev),
+               "V_out": torch.empty((c.B, c.H_kv, L_R, c.D), dtype=self.dtype, device=dev),
+               "idx": torch.empty((c.B, c.H_kv, L_R), dtype=torch.int32, device=dev)}
+        if want_scores:
+            out["scores"] = torch.empty((c.B, c.H_kv, n_c, c.lag), dtype=torch.float32, device=dev)
+        rc = self.lib.lagkv_compress_prefill_paged(
+            self.handle, _ptr(K_pool), _ptr(V_pool), ctypes.byref(lay), int(S_in), _ptr(out["K_out"]),
+            _ptr(out["V_out"]), _ptr(out["idx"]), _ptr(out.get("scores")), _ptr(workspace), workspace.numel(),
+            _stream(dev))
+        _check(rc, "lagkv_compress_prefill_paged")
+        out["L_R"], out["n_c"] = L_R, n_c
+        return out
+
+    def compress_append_paged(self, K_pool, V_pool, block_table, seq_len, static_len, workspace, max_new_chunks=1,
+                              idx_out=None, scores_out=None, strides=None):
+        """``lagkv_compress_append_paged``: in place inside the sequences' own pages."""
+        self._check_cache(K_pool, "K_pool")
+        self._check_cache(V_pool, "V_pool")
+        lay = self._paged(K_pool, block_table, strides)
+        rc = self.lib.lagkv_compress_append_paged(
+            self.handle, _ptr(K_pool), _ptr(V_pool), ctypes.byref(lay), _ptr(seq_len), _ptr(static_len),
+            int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(workspace), workspace.numel(),
+            _stream(self._dev()))
+        _check(rc, "lagkv_compress_append_paged")
 
     def gather(self, K, V, idx, workspace=None, S_in=None):
         """``lagkv_gather``: rows ``idx`` ``[B, H, n_idx]`` int32 of K (and V, may be None)."""

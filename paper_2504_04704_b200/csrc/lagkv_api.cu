@@ -233,19 +233,18 @@ int choose_shape(lagkv_plan_s* pl) {
     pl->tuned = false;
     pl->app_tuned = false;
     pl->app_pair.kidx = -1;
-    // one-partition appends (decode): the smallest cluster whose CTAs keep the whole window
-    // resident with two CTAs to an SM, else the pair of CTAs with as much of it as fits
+    // One-partition appends (decode).  Measured on the decode workload (L = 512, k = 128): a CTA's
+    // chain of dependent steps (loads, two exchanges, selection, gather, stores) takes 15-20 us
+    // whatever its share, so clusters only pay while the GPU is not full: with 64 units a cluster
+    // of four per unit takes 32 us against 50 us for one CTA per unit, with 128 units a pair
+    // 38 us against 42-50 us; from 256 units on the uniform kernel (two large CTAs per SM) wins.
     if (pl->cfg.variant == LAGKV_VARIANT_LAGKV) {
-        bool found = false;
-        for (int splits = 1; splits <= kAppendMaxSplits && !found; splits *= 2) {
-            const int rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, splits, 2, 2, true);
-            if (rc2 == LAGKV_ECUDA) return rc2;
-            found = rc2 == LAGKV_OK;
-        }
-        if (!found) {
-            const int rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, 1, 2, 1, false);
-            if (rc2 == LAGKV_ECUDA) return rc2;
-        }
+        const long long U = (long long)pl->cfg.B * pl->cfg.H_kv;
+        int rc2 = LAGKV_EUNSUPPORTED;
+        if (2 * U <= pl->sm_count) rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, 2, 2, 2, true);
+        if (rc2 == LAGKV_EUNSUPPORTED && U <= pl->sm_count)
+            rc2 = make_append_cluster(pl, LAGKV_TUNE_APPEND_CLUSTER, 1, 2, 2, false);
+        if (rc2 == LAGKV_ECUDA) return rc2;
     }
     if (L >= 256) {
         const Cand ws[] = {{12, 32, 2, 1}, {12, 16, 3, 1}, {12, 16, 2, 1}};
@@ -277,7 +276,54 @@ const Shape& prefill_shape(const lagkv_plan_s* pl, long long slots) {
 
 struct Strides {
     long long sb, sh, ss;
+    // paged caches: block table and page geometry (block_table == nullptr: not paged)
+    const int32_t* block_table = nullptr;
+    long long page_stride = 0;
+    int max_blocks = 0, page_shift = 0;
 };
+// Checks a paged layout and turns it into strides; S is the number of rows the call addresses.
+int resolve_paged(const lagkv_config& c, const lagkv_paged_layout* lay, int64_t S, Strides* out) {
+    if (lay == nullptr || lay->block_table == nullptr || (reinterpret_cast<uintptr_t>(lay->block_table) & 3u))
+        return LAGKV_EINVAL;
+    if (c.stride_b != 0 || c.stride_h != 0 || c.stride_s != 0) return LAGKV_EINVAL;  // the layout carries the strides
+    const int ps = lay->page_size;
+    if (ps < 16 || ps > (1 << 20) || (ps & (ps - 1)) != 0 || lay->max_blocks < 1) return LAGKV_EINVAL;
+    if ((long long)lay->max_blocks * ps < S) return LAGKV_EINVAL;
+    long long ss = lay->stride_s ? lay->stride_s : c.D;
+    long long sh = lay->stride_h ? lay->stride_h : (long long)ps * ss;
+    long long sp = lay->stride_page ? lay->stride_page : (long long)c.H_kv * sh;
+    if (ss < c.D || (ss % 8) || (sh % 8) || (sp % 8) || sh < 0 || sp <= 0) return LAGKV_EINVAL;
+    out->sb = 0;
+    out->sh = sh;
+    out->ss = ss;
+    out->block_table = lay->block_table;
+    out->page_stride = sp;
+    out->max_blocks = lay->max_blocks;
+    out->page_shift = 0;
+    while ((1 << out->page_shift) < ps) ++out->page_shift;
+    return LAGKV_OK;
+}
+CacheLayout cache_layout(const Strides& st, int H) {
+    CacheLayout l;
+    l.sb = st.sb;
+    l.sh = st.sh;
+    l.ss = st.ss;
+    l.page_stride = st.page_stride;
+    l.block_table = st.block_table;
+    l.H = H;
+    l.max_blocks = st.max_blocks;
+    l.page_shift = st.page_shift;
+    return l;
+}
+void set_layout(Params& P, const Strides& st) {
+    P.sb = st.sb;
+    P.sh = st.sh;
+    P.ss = st.ss;
+    P.block_table = st.block_table;
+    P.page_stride = st.page_stride;
+    P.max_blocks = st.max_blocks;
+    P.page_shift = st.page_shift;
+}
 int resolve_strides(const lagkv_config& c, int64_t S, Strides* out) {
     long long ss = c.stride_s ? c.stride_s : c.D;
     long long sh = c.stride_h ? c.stride_h : (long long)S * ss;
@@ -427,7 +473,7 @@ int lagkv_workspace_init(lagkv_plan_t plan, void* workspace, size_t workspace_by
 // lagkv_compress_prefill() for the first B sequences of the plan (the host pipeline runs it chunk by chunk)
 static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, int64_t S_in, void* K_out,
                         void* V_out, int32_t* idx_out, float* scores_out, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream) {
+                        size_t workspace_bytes, void* cuda_stream, const lagkv_paged_layout* paged = nullptr) {
     if (plan == nullptr || K == nullptr || V == nullptr || plan->cfg.device < 0) return LAGKV_EINVAL;
     if ((K_out == nullptr) != (V_out == nullptr)) return LAGKV_EINVAL;
     if (S_in < 0 || S_in > 0x7fffffffll - 65536) return LAGKV_EINVAL;
@@ -439,7 +485,11 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LAGKV_EINVAL;
     const lagkv_config& c = plan->cfg;
     Strides st;
-    if (resolve_strides(c, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    if (paged != nullptr) {
+        if (resolve_paged(c, paged, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    } else if (resolve_strides(c, S_in, &st) != LAGKV_OK) {
+        return LAGKV_EINVAL;
+    }
     if (S_in == 0) return LAGKV_OK;
 
     DeviceGuard guard(c.device);
@@ -454,7 +504,7 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
         const long long want = (total + block - 1) / block;
         const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
         lagkv_copy_kernel<<<grid, block, 0, stream>>>(
-            static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), st.sb, st.sh, st.ss, c.H_kv,
+            static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), cache_layout(st, c.H_kv),
             int(S_in), c.D / 8, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), idx_out, U);
         return check_launch();
     }
@@ -468,9 +518,7 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
     P.idx_out = idx_out;
     P.scores_out = scores_out;
     P.status = static_cast<int32_t*>(workspace);
-    P.sb = st.sb;
-    P.sh = st.sh;
-    P.ss = st.ss;
+    set_layout(P, st);
     P.B = B;
     P.H = c.H_kv;
     P.L = c.lag;
@@ -485,7 +533,9 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
     P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : (c.variant == LAGKV_VARIANT_L2NORM ? P.n - 1 : P.n);
     P.total_slots = U * P.spu;
-    const Shape& shape = prefill_shape(plan, P.total_slots);
+    // paged caches go through the uniform kernel (the only family that looks rows up page by page)
+    const Shape& shape = paged != nullptr ? (kKernels[plan->pre.kidx].ws ? plan->app : plan->pre)
+                                          : prefill_shape(plan, P.total_slots);
     P.stages = shape.stages;
     // Measured on the Ls = 65536 sweep and the 32K / 128K configurations: with L >= 1024 and
     // 1/8 <= k/L <= 1/4 the select warps gain 2-7 % by moving every second partition's kept rows;
@@ -636,14 +686,15 @@ static int append_check(lagkv_plan_t plan, const void* K_cache, const void* V_ca
     return LAGKV_OK;
 }
 
-int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
-                          int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
-                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static int append_impl(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
+                       int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream, const lagkv_paged_layout* paged) {
     Strides st;
     const int chk = append_check(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out,
                                  scores_out, workspace, workspace_bytes, &st);
     if (chk != LAGKV_OK) return chk;
     const lagkv_config& c = plan->cfg;
+    if (paged != nullptr && resolve_paged(c, paged, S_cap, &st) != LAGKV_OK) return LAGKV_EINVAL;
 
     DeviceGuard guard(c.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -659,9 +710,7 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     P.status = static_cast<int32_t*>(workspace);
     P.seq_done = static_cast<int32_t*>(workspace) + kStatusWords;
     P.kept_pos = idx_out ? idx_out : P.seq_done + counter_words(plan);
-    P.sb = st.sb;
-    P.sh = st.sh;
-    P.ss = st.ss;
+    set_layout(P, st);
     P.B = c.B;
     P.H = c.H_kv;
     P.L = c.lag;
@@ -676,7 +725,7 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
 
     const long long U = (long long)c.B * c.H_kv;
     void* args[] = {&P};
-    if (max_new_chunks == 1 && plan->app_pair.kidx >= 0 && !plan->app_tuned) {
+    if (max_new_chunks == 1 && plan->app_pair.kidx >= 0 && !plan->app_tuned && paged == nullptr) {
         // decode: at most one partition per sequence and call -> a cluster of CTAs per unit
         const KernelEntry& kp = kKernels[plan->app_pair.kidx];
         P.idx_out = idx_out;
@@ -706,6 +755,31 @@ int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64
     return check_launch();
 }
 
+int lagkv_compress_append(lagkv_plan_t plan, void* K_cache, void* V_cache, int64_t S_cap, int32_t* seq_len,
+                          int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out, float* scores_out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return append_impl(plan, K_cache, V_cache, S_cap, seq_len, static_len, max_new_chunks, idx_out, scores_out,
+                       workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+int lagkv_compress_prefill_paged(lagkv_plan_t plan, const void* K_pool, const void* V_pool,
+                                 const lagkv_paged_layout* layout, int64_t S_in, void* K_out, void* V_out,
+                                 int32_t* idx_out, float* scores_out, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream) {
+    if (plan == nullptr || layout == nullptr) return LAGKV_EINVAL;
+    return prefill_impl(plan, plan->cfg.B, K_pool, V_pool, S_in, K_out, V_out, idx_out, scores_out, workspace,
+                        workspace_bytes, cuda_stream, layout);
+}
+
+int lagkv_compress_append_paged(lagkv_plan_t plan, void* K_pool, void* V_pool, const lagkv_paged_layout* layout,
+                                int32_t* seq_len, int32_t* static_len, int32_t max_new_chunks, int32_t* idx_out,
+                                float* scores_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (plan == nullptr || layout == nullptr || layout->page_size < 1 || layout->max_blocks < 1) return LAGKV_EINVAL;
+    const int64_t S_cap = (int64_t)layout->max_blocks * layout->page_size;  // rows a sequence's table can address
+    return append_impl(plan, K_pool, V_pool, S_cap, seq_len, static_len, max_new_chunks, idx_out, scores_out,
+                       workspace, workspace_bytes, cuda_stream, layout);
+}
+
 int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, const int32_t* idx, int64_t n_idx,
                  void* K_out, void* V_out, void* workspace, void* cuda_stream) {
     if (plan == nullptr || K == nullptr || K_out == nullptr || idx == nullptr || plan->cfg.device < 0)
@@ -726,7 +800,7 @@ int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, 
     const long long want = (total + block - 1) / block;
     const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
     lagkv_gather_kernel<<<grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), st.sb, st.sh, st.ss, c.H_kv, int(S_in),
+        static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), cache_layout(st, c.H_kv), int(S_in),
         c.D / 8, idx, n_idx, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), U,
         static_cast<int32_t*>(workspace));
     return check_launch();

@@ -53,7 +53,54 @@ struct Params {
     int stages;                   // ring depth per warp
     int sel_emit;                 // warp-specialised kernel: select warps move the kept rows of odd slots
     int res_tiles;                // append pair kernel: tiles of the window that stay in shared memory
+    // paged caches (uniform kernel, gather): K / V point at a pool of pages, a sequence's rows
+    // [j * page, (j + 1) * page) live in page block_table[b * max_blocks + j]; sh and ss are the
+    // head and row strides inside a page, sb is unused
+    const int32_t* block_table;   // device [B, max_blocks]; nullptr = not paged
+    long long page_stride;        // elements between pages
+    int max_blocks;
+    int page_shift;               // rows per page = 1 << page_shift
 };
+
+// Where the rows of one (b, h) unit live: element offset of row r from the tensor's base pointer.
+// Contiguous caches: base + r * ss.  Paged caches: page lookup, then head and row inside the page.
+struct RowMap {
+    long long base;        // offset of the unit (contiguous) or of the head inside a page (paged)
+    long long ss;          // row stride
+    const int32_t* pages;  // this sequence's row of the block table; nullptr = not paged
+    long long page_stride;
+    int page_shift;
+    __device__ __forceinline__ long long off(int row) const {
+        if (pages == nullptr) return base + (long long)row * ss;
+        return (long long)__ldg(pages + (row >> page_shift)) * page_stride + base +
+               (long long)(row & ((1 << page_shift) - 1)) * ss;
+    }
+    // how many rows starting at `row` are laid out one after another (up to the end of its page)
+    __device__ __forceinline__ int run(int row) const {
+        return pages == nullptr ? 0x40000000 : (1 << page_shift) - (row & ((1 << page_shift) - 1));
+    }
+};
+__device__ __forceinline__ RowMap make_rowmap(const Params& P, int u) {
+    RowMap m;
+    const int b = u / P.H, h = u % P.H;
+    m.ss = P.ss;
+    m.page_stride = P.page_stride;
+    m.page_shift = P.page_shift;
+    if (P.block_table == nullptr) {
+        m.pages = nullptr;
+        m.base = (long long)b * P.sb + (long long)h * P.sh;
+    } else {
+        m.pages = P.block_table + (long long)b * P.max_blocks;
+        m.base = (long long)h * P.sh;
+    }
+    return m;
+}
+// rows [row0, row0 + rows) of a unit -> shared memory at dst, completing on bar, as few bulk
+// copies as the layout allows (lane 0 alone when rows are dense, else one row per lane).
+// The expect_tx for all of it must already be posted.  Warp-collective.
+__device__ __forceinline__ void fetch_rows(const uint16_t* X, const RowMap& m, int row0, int rows, uint32_t dst,
+                                           uint32_t bar, uint32_t rowb, bool dense, int lane);
+
 
 // ------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -214,6 +261,37 @@ __device__ __forceinline__ f32x2 widen2(uint32_t w) {
 
 __device__ __forceinline__ uint4 ld_nc(const uint4* p) { return __ldg(p); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ void fetch_rows(const uint16_t* X, const RowMap& m, int row0, int rows, uint32_t dst,
+                                           uint32_t bar, uint32_t rowb, bool dense, int lane) {
+    if (dense) {
+        if (lane == 0) {
+            for (int r = 0; r < rows;) {
+                const int seg = min(rows - r, m.run(row0 + r));
+                bulk_g2s(dst + uint32_t(r) * rowb, X + m.off(row0 + r), uint32_t(seg) * rowb, bar);
+                r += seg;
+            }
+        }
+    } else {
+        __syncwarp();
+        for (int r = lane; r < rows; r += 32) bulk_g2s(dst + uint32_t(r) * rowb, X + m.off(row0 + r), rowb, bar);
+    }
+}
+// the reverse: shared memory -> rows [row0, row0 + rows) of a unit (bulk-group stores; the caller commits)
+__device__ __forceinline__ void store_rows(uint16_t* X, const RowMap& m, int row0, int rows, uint32_t src, uint32_t rowb,
+                                           bool dense, int lane) {
+    if (dense) {
+        if (lane == 0) {
+            for (int r = 0; r < rows;) {
+                const int seg = min(rows - r, m.run(row0 + r));
+                bulk_s2g(X + m.off(row0 + r), src + uint32_t(r) * rowb, uint32_t(seg) * rowb);
+                r += seg;
+            }
+        }
+    } else {
+        for (int r = lane; r < rows; r += 32) bulk_s2g(X + m.off(row0 + r), src + uint32_t(r) * rowb, rowb);
+    }
+}
 
 __device__ __forceinline__ void record_status(int32_t* status, int code, int detail) {
     if (status != nullptr && atomicCAS(status, 0, code) == 0) status[1] = detail;
@@ -800,7 +878,7 @@ __device__ __forceinline__ void score_and_select(float* sg0, float* sg1, int L, 
 // dst rows [dst_row0, +nrows) <- src rows [src_row0, +nrows), both tensors, disjoint buffers.
 template <int NT, int VPR>
 __device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
-                          long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
+                          const RowMap& m, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
                           int src_row0, int dst_row0, int nrows, int32_t* __restrict__ idx_dst, int tid) {
     if (dstK != nullptr) {
         const long long items = (long long)nrows * 2 * VPR;
@@ -815,7 +893,7 @@ __device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __r
                     const long long r2 = i / VPR;
                     const int row = int(r2 >> 1);
                     const uint16_t* s = (r2 & 1) ? srcV : srcK;
-                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + (src_row0 + row) * ss) + vec);
+                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + m.off(src_row0 + row)) + vec);
                 }
             }
 #pragma unroll
@@ -838,14 +916,14 @@ __device__ void copy_rows(const uint16_t* __restrict__ srcK, const uint16_t* __r
 // kept rows of one partition -> output (prefill, out of place)
 template <int NT, int VPR, int U = 4, bool PREFETCH = false>
 __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __restrict__ srcV,
-                          long long ss, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
+                          const RowMap& m, uint16_t* __restrict__ dstK, uint16_t* __restrict__ dstV,
                           int src_row0, int dst_row0, const int* __restrict__ kept, int k,
                           int32_t* __restrict__ idx_dst, int tid) {
     if (dstK != nullptr) {
         if (PREFETCH) {  // put every kept row in flight towards L2 before the first load waits
             for (int j = tid; j < 2 * k; j += NT) {
                 const uint16_t* s = (j & 1) ? srcV : srcK;
-                prefetch_l2(s + (long long)(src_row0 + kept[j >> 1]) * ss, VPR * 16);
+                prefetch_l2(s + m.off(src_row0 + kept[j >> 1]), VPR * 16);
             }
         }
         const int items = k * 2 * VPR;
@@ -857,7 +935,7 @@ __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __r
                 if (i < items) {
                     const int vec = i % VPR, r2 = i / VPR, j = r2 >> 1;
                     const uint16_t* s = (r2 & 1) ? srcV : srcK;
-                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + (long long)(src_row0 + kept[j]) * ss) + vec);
+                    buf[u] = ld_nc(reinterpret_cast<const uint4*>(s + m.off(src_row0 + kept[j])) + vec);
                 }
             }
 #pragma unroll
@@ -881,15 +959,16 @@ __device__ void emit_kept(const uint16_t* __restrict__ srcK, const uint16_t* __r
 // and destinations both ascend and src >= dst for every j, so when chunks of R rows are taken
 // in order, what a chunk overwrites lies below everything a later chunk reads: the load of
 // chunk c+1 may be in flight while chunk c is stored.  Two stages of R rows of K and R rows of
-// V in shared memory (the tile rings, idle by now), one mbarrier each.  Returns false when a
-// bounded wait ran out.
+// V in shared memory (the tile rings, idle by now), one mbarrier each.  K and V are the
+// tensors' base pointers, m says where the unit's rows are (contiguous or paged).  Returns
+// false when a bounded wait ran out.
 template <class G>
-__device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, long long ss, int dst_row0, int total, int n_kept,
+__device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, const RowMap& m, int dst_row0, int total, int n_kept,
                                const int32_t* kept_pos, int win_src0, uint32_t stage0, int R,
                                uint32_t bar0, int lane) {
     constexpr uint32_t ROWB = G::D * 2;
     const uint32_t stage_bytes = 2u * uint32_t(R) * ROWB;
-    const bool contiguous = ss == G::D;
+    const bool dense = m.ss == G::D;
     const int nchunks = (total + R - 1) / R;
     auto load = [&](int c) {
         const int j0 = c * R, nr = min(R, total - j0);
@@ -900,16 +979,13 @@ __device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, long long ss, int dst_r
             mbar_arrive_expect_tx(bar, 2u * uint32_t(nr) * ROWB);
         }
         __syncwarp();
-        if (contiguous && j0 >= n_kept) {  // window rows: one copy per tensor
-            if (lane == 0) {
-                const long long src = (long long)(win_src0 + j0) * ss;
-                bulk_g2s(dK, K + src, uint32_t(nr) * ROWB, bar);
-                bulk_g2s(dV, V + src, uint32_t(nr) * ROWB, bar);
-            }
+        if (dense && j0 >= n_kept) {  // window rows: as few copies per tensor as the layout allows
+            fetch_rows(K, m, win_src0 + j0, nr, dK, bar, ROWB, true, lane);
+            fetch_rows(V, m, win_src0 + j0, nr, dV, bar, ROWB, true, lane);
         } else {
             for (int r = lane; r < nr; r += 32) {
                 const int j = j0 + r;
-                const long long src = (long long)(j < n_kept ? kept_pos[j] : win_src0 + j) * ss;
+                const long long src = m.off(j < n_kept ? kept_pos[j] : win_src0 + j);
                 bulk_g2s(dK + uint32_t(r) * ROWB, K + src, ROWB, bar);
                 bulk_g2s(dV + uint32_t(r) * ROWB, V + src, ROWB, bar);
             }
@@ -919,19 +995,8 @@ __device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, long long ss, int dst_r
         const int j0 = c * R, nr = min(R, total - j0);
         const uint32_t sK = stage0 + uint32_t(c & 1) * stage_bytes, sV = sK + uint32_t(R) * ROWB;
         if (!mbar_wait_bounded(bar0 + 8 * (c & 1), uint32_t(c >> 1) & 1u)) return false;
-        if (contiguous) {
-            if (lane == 0) {
-                const long long dst = (long long)(dst_row0 + j0) * ss;
-                bulk_s2g(K + dst, sK, uint32_t(nr) * ROWB);
-                bulk_s2g(V + dst, sV, uint32_t(nr) * ROWB);
-            }
-        } else {
-            for (int r = lane; r < nr; r += 32) {
-                const long long dst = (long long)(dst_row0 + j0 + r) * ss;
-                bulk_s2g(K + dst, sK + uint32_t(r) * ROWB, ROWB);
-                bulk_s2g(V + dst, sV + uint32_t(r) * ROWB, ROWB);
-            }
-        }
+        store_rows(K, m, dst_row0 + j0, nr, sK, ROWB, dense, lane);
+        store_rows(V, m, dst_row0 + j0, nr, sV, ROWB, dense, lane);
         bulk_commit();  // every lane closes a group (empty for the lanes that stored nothing)
         return true;
     };
@@ -1023,9 +1088,6 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     auto slot_unit = [&](long long s) -> int { return P.mode == MODE_PREFILL ? int(s / spu) : unit_fixed; };
     auto slot_part = [&](long long s) -> int { return part_of(int(s % spu)); };
     const uint16_t* tbase = tensor ? P.V : P.K;
-    auto unit_base = [&](const uint16_t* base, int u) -> const uint16_t* {
-        return base + (long long)(u / P.H) * P.sb + (long long)(u % P.H) * P.sh;
-    };
 
     // ---- per-warp ring
     const uint32_t ring_w = smem_u32(ring) + uint32_t(warp) * NS * G::TILE_BYTES;
@@ -1045,26 +1107,24 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     long long ps = s_lo;  // producer cursor: next tile to request
     int pt = wj;
     int pslot = 0;
+    int pmap_u = -1;      // unit the producer's row map is for
+    RowMap pmap;
     auto issue_next = [&]() {  // warp-collective
         if (!has_tiles || ps >= s_hi) return;
         const int u = slot_unit(ps), p = slot_part(ps);
+        if (u != pmap_u) {
+            pmap = make_rowmap(P, u);
+            pmap_u = u;
+        }
         const int row0 = stat_rows + p * L + pt * G::TR;
         const int rows = min(G::TR, L - pt * G::TR);
-        const uint16_t* src = unit_base(tbase, u) + (long long)row0 * P.ss;
         const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
         const uint32_t bar = bar_w + 8 * pslot;
-        const uint32_t bytes = uint32_t(rows) * G::D * 2;
         if (lane == 0) {
             fence_proxy_async();
-            mbar_arrive_expect_tx(bar, bytes);
+            mbar_arrive_expect_tx(bar, uint32_t(rows) * G::D * 2);
         }
-        if (contiguous) {
-            if (lane == 0) bulk_g2s(dst, src, bytes, bar);
-        } else {
-            __syncwarp();
-            for (int r = lane; r < rows; r += 32)
-                bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
-        }
+        fetch_rows(tbase, pmap, row0, rows, dst, bar, G::D * 2, contiguous, lane);
         pt += G::WT;
         if (pt >= ntiles) {
             pt = wj;
@@ -1165,7 +1225,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
                                      [] { __syncthreads(); }, [] {});
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {
-                emit_kept<G::NT, G::VPR>(unit_base(P.K, u), unit_base(P.V, u), P.ss,
+                emit_kept<G::NT, G::VPR>(P.K, P.V, make_rowmap(P, u),
                                          P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr,
                                          P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr,
                                          stat_rows + p * L, stat_rows + p * k, kept, k,
@@ -1186,15 +1246,14 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
 
         // ---- rows copied verbatim (prefill): window with a unit's first slot, sink with its last
         if (P.mode == MODE_PREFILL && s >= s_first) {
-            const uint16_t* uk = unit_base(P.K, u);
-            const uint16_t* uv = unit_base(P.V, u);
+            const RowMap um = make_rowmap(P, u);
             uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
             uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
             int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
             if (first_of_unit)
-                copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, stat_rows + (n - 1) * L, stat_rows + (n - 1) * k,
+                copy_rows<G::NT, G::VPR>(P.K, P.V, um, ok, ov, stat_rows + (n - 1) * L, stat_rows + (n - 1) * k,
                                          L + P.rem, oi, tid);
-            if (last_of_unit) copy_rows<G::NT, G::VPR>(uk, uv, P.ss, ok, ov, 0, 0, stat_rows, oi, tid);
+            if (last_of_unit) copy_rows<G::NT, G::VPR>(P.K, P.V, um, ok, ov, 0, 0, stat_rows, oi, tid);
         }
         if (last_of_unit) have_ref = false;  // next slot belongs to another unit
         __syncthreads();
@@ -1203,13 +1262,13 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     // ---- append: pack kept rows behind the static part, then slide the window down
     if (P.mode == MODE_APPEND) {
         const int u = unit_fixed;
-        uint16_t* ck = const_cast<uint16_t*>(unit_base(P.K, u));
-        uint16_t* cv = const_cast<uint16_t*>(unit_base(P.V, u));
+        uint16_t* ck = const_cast<uint16_t*>(P.K);
+        uint16_t* cv = const_cast<uint16_t*>(P.V);
         const int n_c = n - 1;
         const int32_t* kp = P.kept_pos + (long long)u * P.max_chunks * k;
         if (!aborted && k < L && warp == 0) {  // kept rows, then the window, as one ascending sequence of rows
             const int R = int(smem_ring_bytes<G>(NS) / (4 * G::D * 2));
-            if (!move_rows_bulk<G>(ck, cv, P.ss, stat_rows, n_c * k + L + rem, n_c * k, kp,
+            if (!move_rows_bulk<G>(ck, cv, make_rowmap(P, u), stat_rows, n_c * k + L + rem, n_c * k, kp,
                                    stat_rows + n_c * L - n_c * k, smem_u32(ring), R, smem_u32(move_bars), lane)) {
                 timed_out = true;
                 if (lane == 0) record_status(P.status, ST_ETIMEOUT, blockIdx.x);

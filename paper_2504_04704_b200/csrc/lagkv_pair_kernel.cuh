@@ -339,8 +339,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             // the flag is raised before the arrival that completes the phase waited for above
             if (!dead && __shfl_sync(0xffffffffu, gave_up[pair], 0) != 0) dead = true;
             const uint32_t ebar = empty_bar + 8 * buf;
-            const uint16_t* uk = unit_base(P.K, u);
-            const uint16_t* uv = unit_base(P.V, u);
+            const RowMap um = make_rowmap(P, u);
             uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
             uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
             int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
@@ -350,15 +349,15 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
                 select_in_warp_dispatch(sg0, sg0 + Lp, L, k, scores_g, kept, lane, [&] {
                     if (lane == 0) mbar_arrive(ebar);  // the sigma buffer goes back to the streamers
                 });
-                emit_kept<32, G::VPR, 8>(uk, uv, P.ss, ok, ov, sink + p * L, sink + p * k, kept, k, oi, lane);
+                emit_kept<32, G::VPR, 8>(P.K, P.V, um, ok, ov, sink + p * L, sink + p * k, kept, k, oi, lane);
                 __syncwarp();  // kept[] is rewritten by the next selection
             } else if (lane == 0) {
                 mbar_arrive(ebar);
             }
             // rows copied verbatim: the window with the unit's top slot, the sink with slot p = 0
             if (s >= s_first && !dead) {
-                if (top) copy_rows<32, G::VPR>(uk, uv, P.ss, ok, ov, sink + (n - 1) * L, sink + (n - 1) * k, L + P.rem, oi, lane);
-                if (p == 0) copy_rows<32, G::VPR>(uk, uv, P.ss, ok, ov, 0, 0, sink, oi, lane);
+                if (top) copy_rows<32, G::VPR>(P.K, P.V, um, ok, ov, sink + (n - 1) * L, sink + (n - 1) * k, L + P.rem, oi, lane);
+                if (p == 0) copy_rows<32, G::VPR>(P.K, P.V, um, ok, ov, 0, 0, sink, oi, lane);
             }
         }
     }

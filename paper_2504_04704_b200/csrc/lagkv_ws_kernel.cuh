@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 // warp and the gather phase).  Every second slot is what they can carry without
                 // holding up the streamers; with short partitions they have no time to spare.
                 if (sel_moves(i) && P.K_out != nullptr)
-                    emit_kept<kWsSelThreads, G::VPR, 16>(unit_base(P.K, u), unit_base(P.V, u), P.ss,
+                    emit_kept<kWsSelThreads, G::VPR, 16>(P.K, P.V, make_rowmap(P, u),
                                                          P.K_out + (long long)u * P.L_R * G::D,
                                                          P.V_out + (long long)u * P.L_R * G::D, sink + p * L,
                                                          sink + p * k, kept, k, nullptr, etid);

@@ -488,6 +488,130 @@ def test_gather(binding, oracle):
     assert plan.read_status(ws)[0] == binding.LAGKV_EINVAL
 
 
+# ----------------------------------------------------------------------------- paged caches
+def paginate(K, V, page_size, extra_pages=3, seed=0, pad=0):
+    """Scatter contiguous caches ``[B, H, S, D]`` over pools ``[num_pages, H, page_size, D (+ pad)]`` in a
+    random page order; returns (K_pool, V_pool, block_table [B, max_blocks] int32).  Unused pool
+    rows hold a marker value; unused table entries name page 0 (never dereferenced)."""
+    B, H, S, D = K.shape
+    nb = (S + page_size - 1) // page_size
+    g = torch.Generator().manual_seed(seed)
+    num_pages = B * nb + extra_pages
+    perm = torch.randperm(num_pages, generator=g)[:B * nb].reshape(B, nb).to(torch.int32)
+    Kp = torch.full((num_pages, H, page_size, D + pad), 9.0, dtype=K.dtype, device=K.device)
+    Vp = torch.full_like(Kp, 9.0)
+    for b in range(B):
+        for j in range(nb):
+            r0, r1 = j * page_size, min(S, (j + 1) * page_size)
+            Kp[perm[b, j], :, :r1 - r0, :D] = K[b, :, r0:r1]
+            Vp[perm[b, j], :, :r1 - r0, :D] = V[b, :, r0:r1]
+    table = torch.zeros((B, nb + 2), dtype=torch.int32)
+    table[:, :nb] = perm
+    return Kp, Vp, table.to(K.device)
+
+
+def unpaginate(Kp, table, S, D):
+    """The contiguous view ``[B, H, S, D]`` of a paged cache."""
+    B, ps = table.shape[0], Kp.shape[2]
+    nb = (S + ps - 1) // ps
+    rows = Kp[table[:, :nb].long()]                       # [B, nb, H, ps, D+pad]
+    return rows.permute(0, 2, 1, 3, 4).reshape(B, Kp.shape[1], nb * ps, -1)[:, :, :S, :D].contiguous()
+
+
+@pytest.mark.parametrize("D,L,k,page,pad,dtype,variant", [
+    (128, 128, 32, 16, 0, torch.bfloat16, 0), (128, 100, 25, 64, 0, torch.bfloat16, 0),
+    (128, 512, 128, 128, 8, torch.bfloat16, 0), (128, 1024, 256, 32, 0, torch.float16, 0),
+    (64, 64, 16, 16, 0, torch.bfloat16, 0), (96, 256, 64, 64, 0, torch.float16, 0), (256, 300, 75, 256, 0, torch.bfloat16, 0),
+    (128, 128, 32, 32, 0, torch.bfloat16, 1), (128, 256, 64, 16, 0, torch.bfloat16, 2)])
+def test_paged_prefill(binding, oracle, D, L, k, page, pad, dtype, variant):
+    """Prefill from a paged cache (random page order, tiles straddling page boundaries because the
+    sink is not a multiple of the tile height) equals the oracle on the contiguous cache."""
+    B, H, sink = 3, 2, 20
+    S = sink + 6 * L + L // 3
+    K, V = synth.make_kv(B, H, S, D, seed=D + L + page, device="cuda:0", dtype=dtype)
+    Kp, Vp, table = paginate(K, V, page, seed=L, pad=pad)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0, dtype=dtype)
+    ws = plan.new_workspace()
+    strides = None if pad == 0 else (H * page * (D + pad), page * (D + pad), D + pad, page)
+    out = plan.compress_prefill_paged(Kp, Vp, table, S, ws, want_scores=True, strides=strides)
+    assert plan.read_status(ws)[0] == 0
+    host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
+            "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
+    storage = oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16
+    if variant == 2:      # Eq. 16: relative tolerance on the norms; same picks as the contiguous call
+        flat = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0, dtype=dtype)
+        ref = flat.compress_prefill(K, V, ws, want_scores=True)
+        assert torch.equal(ref["idx"], out["idx"]) and torch.equal(ref["K_out"], out["K_out"])
+        assert torch.equal(ref["V_out"], out["V_out"]) and torch.equal(ref["scores"], out["scores"])
+    else:
+        check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host, variant=variant,
+                             storage=storage)
+    # the pools are read-only for a prefill
+    Kp2, Vp2, _ = paginate(K, V, page, seed=L, pad=pad)
+    assert torch.equal(Kp, Kp2) and torch.equal(Vp, Vp2)
+
+
+def test_paged_prefill_identity_and_errors(binding, oracle):
+    B, H, D, sink, L, k, page = 2, 2, 128, 8, 64, 16, 16
+    S = sink + 2 * L - 1                                     # too short: identity
+    K, V = synth.make_kv(B, H, S, D, seed=3, device="cuda:0")
+    Kp, Vp, table = paginate(K, V, page, seed=1)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0)
+    ws = plan.new_workspace()
+    out = plan.compress_prefill_paged(Kp, Vp, table, S, ws)
+    assert out["L_R"] == S and torch.equal(out["K_out"], K) and torch.equal(out["V_out"], V)
+    assert out["idx"][0, 0].tolist() == list(range(S))
+    with pytest.raises(binding.LagKVError):                  # page size not a power of two
+        plan.compress_prefill_paged(Kp, Vp, table, S, ws, strides=(0, 0, 0, 24))
+    with pytest.raises(binding.LagKVError):                  # table too short for S_in rows
+        plan.compress_prefill_paged(Kp, Vp, table[:, :2].contiguous(), S, ws)
+    strided = binding.Plan(B, H, D, sink, L, keep_k=k, strides=(H * S * D, S * D, D), device=0)
+    with pytest.raises(binding.LagKVError):                  # a plan with its own strides cannot take pages
+        strided.compress_prefill_paged(Kp, Vp, table, S, ws)
+
+
+@pytest.mark.parametrize("D,L,k,page,chunks,variant", [(128, 64, 16, 16, 3, 0), (128, 512, 128, 64, 1, 0),
+                                                       (128, 96, 24, 32, 2, 0), (64, 128, 32, 128, 1, 0),
+                                                       (256, 100, 10, 16, 2, 0), (128, 128, 32, 16, 2, 1),
+                                                       (128, 128, 32, 64, 1, 2)])
+def test_paged_append(binding, oracle, D, L, k, page, chunks, variant):
+    """In-place append on a paged cache with a ragged batch (different lengths, one sequence
+    skips): lengths, every valid row and the kept positions equal the oracle's replay on the
+    contiguous cache; rows beyond a sequence's old length and pages of nobody stay untouched."""
+    B, H, sink = 4, 3, 8
+    stat = [sink, sink + 2 * k, sink + k, sink]
+    seq = [stat[0] + (chunks + 1) * L + 3, stat[1] + (chunks + 1) * L, stat[2] + 2 * L + L - 1, stat[3] + 2 * L - 1]
+    S = max(seq) + 5
+    K, V = synth.make_kv(B, H, S, D, seed=D + L + page + chunks, device="cuda:0")
+    Kp, Vp, table = paginate(K, V, page, seed=L + 1)
+    Kp0, Vp0 = Kp.clone(), Vp.clone()
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0)
+    ws = plan.new_workspace(chunks)
+    seq_d = torch.tensor(seq, dtype=torch.int32, device="cuda:0")
+    stat_d = torch.tensor(stat, dtype=torch.int32, device="cuda:0")
+    idx_out = torch.full((B, H, chunks * k), -1, dtype=torch.int32, device="cuda:0")
+    plan.compress_append_paged(Kp, Vp, table, seq_d, stat_d, ws, max_new_chunks=chunks, idx_out=idx_out)
+    assert plan.read_status(ws)[0] == 0
+    Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(synth.to_bits(K), synth.to_bits(V), np.array(seq),
+                                                         np.array(stat), L, k, variant=variant)
+    assert seq_d.tolist() == seq_r.tolist() and stat_d.tolist() == stat_r.tolist()
+    Kg, Vg = synth.to_bits(unpaginate(Kp, table, S, D)), synth.to_bits(unpaginate(Vp, table, S, D))
+    Kb, Vb = synth.to_bits(K), synth.to_bits(V)
+    for b in range(B):
+        n = int(seq_r[b])
+        np.testing.assert_array_equal(Kg[b, :, :n], Kr[b, :, :n])
+        np.testing.assert_array_equal(Vg[b, :, :n], Vr[b, :, :n])
+        np.testing.assert_array_equal(Kg[b, :, seq[b]:], Kb[b, :, seq[b]:])
+        if kept[b].shape[1]:
+            np.testing.assert_array_equal(idx_out[b, :, :kept[b].shape[1]].cpu().numpy(), kept[b])
+    # pages that belong to no sequence, and the rows of a page behind the cache's end, are never written
+    used = torch.zeros(Kp.shape[0], dtype=torch.bool)
+    nb = (S + page - 1) // page
+    used[table[:, :nb].cpu().long().flatten()] = True
+    used = used.to("cuda:0")
+    assert torch.equal(Kp[~used], Kp0[~used]) and torch.equal(Vp[~used], Vp0[~used])
+
+
 # -------------------------------------------------------------------------------- append
 def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chunks, seed, tune=None, give_idx=True,
                 variant=0, dtype=torch.bfloat16):
