@@ -3,6 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
                     [--variant lagkv|localkv|l2norm] [--storage bf16|fp16] [--layers N] [--tune w,t,s,c]
+                    [--paged PAGE_ROWS]
     python bench.py --workload sweep --sweep [--sweep-B 1,8]   # one JSON line per (L, r, B) cell of the sweep
     python bench.py --workload decode_append --append          # the incremental pass, one triggering call per step
     python bench.py --workload decode_append --append --loop [--ragged]
@@ -30,6 +31,7 @@ Beside the contract's keys the default line carries
 from __future__ import annotations
 
 import argparse
+import ctypes
 import datetime
 import hashlib
 import json
@@ -533,6 +535,30 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
            "idx": torch.empty((Bf, w.H, L_R), dtype=torch.int32, device=dev)}
     info = plan.launch_info(w.S)
     step = lambda: plan.compress_prefill(K, V, ws, out=out)
+    if args.paged:
+        # the same cache cut into pages of args.paged rows, scattered over a pool in random order
+        ps = args.paged
+        nb = (w.S + ps - 1) // ps
+        g = torch.Generator().manual_seed(1)
+        perm = torch.randperm(Bf * nb, generator=g).reshape(Bf, nb).to(torch.int32).to(dev)
+        pools = []
+        for X in (K, V):
+            pool = torch.empty((Bf * nb, w.H, ps, w.D), dtype=store, device=dev)
+            padded = X if nb * ps == w.S else torch.nn.functional.pad(X, (0, 0, 0, nb * ps - w.S))
+            for b in range(Bf):        # rows [j*ps, (j+1)*ps) of sequence b -> page perm[b, j]
+                pool[perm[b].long()] = padded[b].reshape(w.H, nb, ps, w.D).permute(1, 0, 2, 3)
+            pools.append(pool)
+            del padded
+        Kp, Vp = pools
+        info = dict(info, kernel=info["paged_kernel"], note="launch shape of the paged call's kernel family")
+
+        def step():
+            rc = plan.lib.lagkv_compress_prefill_paged(
+                plan.handle, binding._ptr(Kp), binding._ptr(Vp), ctypes.byref(lay), w.S, binding._ptr(out["K_out"]),
+                binding._ptr(out["V_out"]), binding._ptr(out["idx"]), None, binding._ptr(ws), ws.numel(),
+                binding._stream(dev))
+            assert rc == 0, rc
+        lay = plan._paged(Kp, perm, None)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -580,6 +606,12 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
 
     # ---- end to end: host cache -> device -> compress -> compacted cache back on the host
     e2e = None
+    if args.paged:      # check the timed launch's result against the contiguous call, then report the pass only
+        ref = plan.compress_prefill(K, V, ws)
+        assert torch.equal(ref["idx"], out["idx"]) and torch.equal(ref["K_out"], out["K_out"])
+        assert torch.equal(ref["V_out"], out["V_out"])
+        del ref
+        full = False
     if full and not args.no_e2e and variant == 0 and args.storage == "bf16":
         chunk = max(1, min(4, w.layers)) * w.B
         while Bf % chunk:
@@ -615,7 +647,7 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
     peak, peak_src = measured_peak()
     alg = algorithmic_bytes(w, L_R, variant)
     achieved = alg / (ms_step * 1e-3) / 1e9
-    captured = not args.layers and not args.tune and variant == 0 and args.storage == "bf16"
+    captured = not args.layers and not args.tune and variant == 0 and args.storage == "bf16" and not args.paged
     traffic = captured_traffic(w.name) if captured else None   # counters of exactly this launch, else null
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -623,7 +655,7 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H_kv": w.H, "D": w.D, "Ls": w.S,
                    "sink": w.sink, "lag": w.lag, "keep_ratio": w.ratio, "keep_k": plan.k, "L_R": L_R,
-                   "variant": args.variant,
+                   "variant": args.variant, "paged": (f"pages of {args.paged} rows, random order" if args.paged else None),
                    "storage": args.storage, "parallelism": f"dp{world} (independent caches per rank, no collective)",
                    "launch": info,
                    "l2": ("inputs (%.2f GB per rank) are far larger than the 126 MB L2; no flush" % (input_bytes / 1e9))
@@ -709,6 +741,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=4096, help="with --append --loop: tokens appended per sequence")
     ap.add_argument("--sweep", action="store_true", help="with --workload sweep: every (L, r) cell, one line each")
     ap.add_argument("--sweep-B", default="1,8", help="batch sizes of the sweep")
+    ap.add_argument("--paged", type=int, default=0, help="read the cache through a block table with pages of N rows")
     ap.add_argument("--sustained", type=float, default=2.0, help="seconds of the sustained run (0 = skip)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

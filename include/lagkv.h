@@ -316,7 +316,8 @@ int lagkv_read_status(lagkv_plan_t plan, void *workspace, void *cuda_stream,
  * Launch shape the plan uses for a prefill of S_in rows: info[0] = grid, info[1] = block
  * threads, info[2] = dynamic shared memory bytes, info[3] = kernel launches per call,
  * info[4] = kernel family (0 = identity copy, 1 = uniform kernel, 2 = warp-specialised
- * kernel, 3 = pair kernel), info[5] = reserved (0).
+ * kernel, 3 = pair kernel), info[5] = kernel family lagkv_compress_prefill_paged() uses for
+ * the same call (1 or 2; 0 for the identity copy).
  */
 int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]);
 

@@ -201,7 +201,9 @@ class Plan:
         info = (ctypes.c_int32 * 6)()
         _check(self.lib.lagkv_launch_info(self.handle, int(S_in), ctypes.byref(info)), "lagkv_launch_info")
         kernel = ("lagkv_copy_kernel", "lagkv_stream_kernel", "lagkv_ws_kernel", "lagkv_pair_kernel")[info[4]]
-        return {"grid": info[0], "block": info[1], "smem": info[2], "launches": info[3], "kernel": kernel}
+        names = ("lagkv_copy_kernel", "lagkv_stream_kernel", "lagkv_ws_kernel", "lagkv_pair_kernel")
+        return {"grid": info[0], "block": info[1], "smem": info[2], "launches": info[3], "kernel": kernel,
+                "paged_kernel": names[info[5]]}
 
     def tune(self, warps=0, tile_rows=0, stages=0, ctas_per_sm=0) -> None:
         _check(self.lib.lagkv_plan_tune(self.handle, int(warps), int(tile_rows), int(stages), int(ctas_per_sm)),

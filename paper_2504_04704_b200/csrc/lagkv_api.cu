@@ -39,6 +39,8 @@ struct KernelTable {
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = append_pair_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = ws_paged_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
     }
 };
 const KernelTable& table() {
@@ -51,10 +53,10 @@ struct KernelRef {  // kKernels[i] reads like an array
 const KernelRef kKernels;
 #define kNumKernels (table().n)
 
-int find_kernel(int D, int NW, int TR, int variant, int dtype) {
+int find_kernel(int D, int NW, int TR, int variant, int dtype, bool paged = false) {
     for (int i = 0; i < kNumKernels; ++i)
         if (kKernels[i].D == D && kKernels[i].NW == NW && kKernels[i].TR == TR && kKernels[i].variant == variant &&
-            kKernels[i].dtype == dtype)
+            kKernels[i].dtype == dtype && kKernels[i].paged == paged)
             return i;
     return -1;
 }
@@ -533,9 +535,22 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
     P.L_R = int(lagkv_compressed_len(plan, S_in, -1));
     P.spu = c.variant == LAGKV_VARIANT_LOCALKV ? 2 * (P.n - 1) : (c.variant == LAGKV_VARIANT_L2NORM ? P.n - 1 : P.n);
     P.total_slots = U * P.spu;
-    // paged caches go through the uniform kernel (the only family that looks rows up page by page)
-    const Shape& shape = paged != nullptr ? (kKernels[plan->pre.kidx].ws ? plan->app : plan->pre)
-                                          : prefill_shape(plan, P.total_slots);
+    // Paged caches: the warp-specialised kernel's paged twin where the plan would use that kernel and
+    // the twin is compiled (same shared memory, so the limit is raised the same way); else the
+    // uniform kernel, which looks rows up page by page in every instantiation.
+    Shape paged_shape;
+    if (paged != nullptr) {
+        paged_shape = kKernels[plan->pre.kidx].ws ? plan->app : plan->pre;
+        const KernelEntry& pre = kKernels[plan->pre.kidx];
+        if (pre.ws && pre.NW != LAGKV_TUNE_PAIRS) {
+            const int twin = find_kernel(pre.D, pre.NW, pre.TR, pre.variant, pre.dtype, true);
+            if (twin >= 0 && raise_smem_limit(reinterpret_cast<const void*>(kKernels[twin].fn), plan->pre.smem)) {
+                paged_shape = plan->pre;
+                paged_shape.kidx = twin;
+            }
+        }
+    }
+    const Shape& shape = paged != nullptr ? paged_shape : prefill_shape(plan, P.total_slots);
     P.stages = shape.stages;
     // Measured on the Ls = 65536 sweep and the 32K / 128K configurations: with L >= 1024 and
     // 1/8 <= k/L <= 1/4 the select warps gain 2-7 % by moving every second partition's kept rows;
@@ -847,7 +862,10 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]) {
     info[3] = 1;
     const KernelEntry& ke = kKernels[shape.kidx];
     info[4] = !ke.ws ? 1 : (ke.NW == LAGKV_TUNE_PAIRS ? 3 : 2);
-    info[5] = 0;
+    // family of the same call on a paged cache: the warp-specialised kernel where its paged twin is
+    // compiled and the plan would use that family, else the uniform kernel
+    const KernelEntry& pre = kKernels[plan->pre.kidx];
+    info[5] = (pre.ws && pre.NW != LAGKV_TUNE_PAIRS && find_kernel(pre.D, pre.NW, pre.TR, pre.variant, pre.dtype, true) >= 0) ? 2 : 1;
     return LAGKV_OK;
 }
 

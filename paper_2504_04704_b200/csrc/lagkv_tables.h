@@ -21,6 +21,7 @@ struct KernelEntry {
     int threads;    // CTA size
     stream_kernel_t fn;
     smem_fn_t smem;
+    bool paged = false;  // reads its caches through a block table (the uniform kernel does both)
 };
 
 // each returns the number of entries and sets *table; the "_dims" tables hold the head
@@ -62,5 +63,10 @@ constexpr int kAppendPairTileRows = 16;
 #define LAGKV_WS_ENTRY_DT(D, V, NWS, TR, DT) \
     LAGKV_WS_ENTRY2(D, V, NWS, TR, 0, DT), LAGKV_WS_ENTRY2(D, V, NWS, TR, 1, DT), LAGKV_WS_ENTRY2(D, V, NWS, TR, 2, DT)
 #define LAGKV_WS_ENTRY(D, V, NWS, TR) LAGKV_WS_ENTRY_DT(D, V, NWS, TR, 0)
+/* the same kernel for paged caches (LagKV scoring) */
+#define LAGKV_WS_PAGED_ENTRY(D, V, NWS, TR, DT) \
+    { D, NWS + kWsEpiWarps, TR, 0, DT, true, (NWS + kWsEpiWarps) * 32, \
+      &lagkv_ws_kernel<Geo<D, V, NWS, TR, DT>, 0, true>, &ws_smem_total_bytes<Geo<D, V, NWS, TR, DT>>, true }
+int ws_paged_kernels(const KernelEntry** table);      // lagkv_ws_kernel reading paged caches
 
 }  // namespace lagkv

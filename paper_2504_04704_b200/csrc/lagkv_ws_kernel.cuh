@@ -51,8 +51,11 @@ __host__ __device__ inline size_t ws_smem_total_bytes(int stages, int L) {
 }
 
 // VAR: 0 = LagKV, 1 = LocalKV, 2 = L2 norm (enum lagkv_variant), compiled apart so that the
-// LagKV kernel carries none of the other variants' code.
-template <class G, int VAR>
+// LagKV kernel carries none of the other variants' code.  PAGED: the caches are pools of pages
+// behind a block table (every row address goes through RowMap; a tile that straddles a page
+// boundary takes two copies); compiled apart too, so that the kernel for contiguous caches keeps
+// its plain pointer arithmetic and its registers.
+template <class G, int VAR, bool PAGED = false>
 __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(const Params P) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -139,12 +142,13 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         long long pleft = s_hi - s_lo;
         int pu = int(s_lo / spu), pj = int(s_lo % spu);
         const uint16_t* pbase = unit_base(tbase, pu);
+        RowMap pmap;  // PAGED only
+        if (PAGED) pmap = make_rowmap(P, pu);
         int pt = wj, pslot = 0;
         auto issue_next = [&]() {  // warp-collective
             if (dead || !has_tiles || pleft <= 0) return;
             const int row0 = sink + slot_part(pj) * L + pt * G::TR;
             const int rows = min(G::TR, L - pt * G::TR);
-            const uint16_t* src = pbase + (long long)row0 * P.ss;
             const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
             const uint32_t bar = bar_w + 8 * pslot;
             const uint32_t bytes = uint32_t(rows) * G::D * 2;
@@ -152,12 +156,17 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar, bytes);
             }
-            if (contiguous) {
-                if (lane == 0) bulk_g2s(dst, src, bytes, bar);
+            if (PAGED) {
+                fetch_rows(tbase, pmap, row0, rows, dst, bar, G::D * 2, contiguous, lane);
             } else {
-                __syncwarp();
-                for (int r = lane; r < rows; r += 32)
-                    bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+                const uint16_t* src = pbase + (long long)row0 * P.ss;
+                if (contiguous) {
+                    if (lane == 0) bulk_g2s(dst, src, bytes, bar);
+                } else {
+                    __syncwarp();
+                    for (int r = lane; r < rows; r += 32)
+                        bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+                }
             }
             pt += WTE;
             if (pt >= ntiles) {  // next slot of this unit, or the first slot of the next unit
@@ -166,7 +175,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 if (++pj == spu) {
                     pj = 0;
                     ++pu;
-                    pbase = unit_base(tbase, pu);
+                    if (PAGED) pmap = make_rowmap(P, pu);
+                    else pbase = unit_base(tbase, pu);
                 }
             }
             if (++pslot == NS) pslot = 0;
@@ -414,12 +424,22 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 }
                 __syncwarp();
                 const uint32_t dK = stage_u32 + uint32_t(2 * st) * CHUNK_BYTES, dV = dK + CHUNK_BYTES;
-                const uint16_t* bK = unit_base(P.K, u);
-                const uint16_t* bV = unit_base(P.V, u);
+                // where the unit's rows are: an offset from the tensor's base pointer
+                RowMap um;
+                if (PAGED) {
+                    um = make_rowmap(P, u);
+                } else {
+                    um.pages = nullptr;
+                    um.ss = P.ss;
+                    um.base = (long long)(u / P.H) * P.sb + (long long)(u % P.H) * P.sh;
+                }
                 if (kind == 1 && contiguous) {
-                    if (lane == 0) {
-                        bulk_g2s(dK, bK + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
-                        bulk_g2s(dV, bV + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                    if (PAGED) {
+                        fetch_rows(P.K, um, src, nr, dK, copy_bar + 8 * st, G::D * 2, true, lane);
+                        fetch_rows(P.V, um, src, nr, dV, copy_bar + 8 * st, G::D * 2, true, lane);
+                    } else if (lane == 0) {
+                        bulk_g2s(dK, P.K + um.base + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                        bulk_g2s(dV, P.V + um.base + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
                     }
                 } else if (lane < nr) {  // one row of K and of V per lane
                     int row = src + lane;
@@ -428,8 +448,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                         row = P.idx_out != nullptr ? __ldcg(P.idx_out + o + lane)
                                                    : __ldcg(reinterpret_cast<const int32_t*>(P.K_out + (o + lane) * G::D));
                     }
-                    bulk_g2s(dK + uint32_t(lane) * G::D * 2, bK + (long long)row * P.ss, G::D * 2, copy_bar + 8 * st);
-                    bulk_g2s(dV + uint32_t(lane) * G::D * 2, bV + (long long)row * P.ss, G::D * 2, copy_bar + 8 * st);
+                    const long long ro = um.off(row);
+                    bulk_g2s(dK + uint32_t(lane) * G::D * 2, P.K + ro, G::D * 2, copy_bar + 8 * st);
+                    bulk_g2s(dV + uint32_t(lane) * G::D * 2, P.V + ro, G::D * 2, copy_bar + 8 * st);
                 }
             }
             if (pending) {  // the chunk loaded before this one goes out
@@ -483,8 +504,10 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         for (long long s = (s_from > s_first ? s_from : s_first); s < s_hi; ++s) {
             const int u = int(s / spu), sj = int(s % spu), p = slot_part(sj);
             if (!slot_scored(sj) || sel_moves(s - s_lo)) continue;  // done by the select warps
-            const uint16_t* srcK = unit_base(P.K, u);
-            const uint16_t* srcV = unit_base(P.V, u);
+            const uint16_t* srcK = PAGED ? P.K : unit_base(P.K, u);
+            const uint16_t* srcV = PAGED ? P.V : unit_base(P.V, u);
+            RowMap um;  // PAGED only
+            if (PAGED) um = make_rowmap(P, u);
             const long long o = (long long)u * P.L_R + sink + p * k;
             uint16_t* dstK = P.K_out + o * G::D;
             uint16_t* dstV = P.V_out + o * G::D;
@@ -510,8 +533,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                         if (src[q][e] >= 0) {
                             const int va = (e * 32 + lane) % RV;
                             const uint16_t* sp = va >= G::VPR ? srcV : srcK;
-                            buf[q][e] = ld_nc(reinterpret_cast<const uint4*>(sp + (long long)src[q][e] * P.ss) +
-                                              (va % G::VPR));
+                            const long long ro = PAGED ? um.off(src[q][e]) : (long long)src[q][e] * P.ss;
+                            buf[q][e] = ld_nc(reinterpret_cast<const uint4*>(sp + ro) + (va % G::VPR));
                         }
 #pragma unroll
                 for (int q = 0; q < UG; ++q)

@@ -551,6 +551,34 @@ def test_paged_prefill(binding, oracle, D, L, k, page, pad, dtype, variant):
     assert torch.equal(Kp, Kp2) and torch.equal(Vp, Vp2)
 
 
+@pytest.mark.parametrize("page,dtype", [(16, torch.bfloat16), (64, torch.float16), (1024, torch.bfloat16)])
+def test_paged_prefill_warp_specialised_many_units(binding, page, dtype):
+    """The warp-specialised kernel's paged twin with several slots per CTA and ranges that start
+    inside a unit: rows, indices and scores are bit-identical to the contiguous call's, with and
+    without the index output (positions parked in the output rows)."""
+    B, H, D, sink, L, k = 8, 5, 128, 16, 256, 64
+    S = sink + 21 * L + 77
+    K, V = synth.make_kv(B, H, S, D, seed=page, device="cuda:0", dtype=dtype)
+    Kp, Vp, table = paginate(K, V, page, seed=page + 1)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0, dtype=dtype)
+    assert plan.launch_info(S)["kernel"] == "lagkv_ws_kernel"
+    ws = plan.new_workspace()
+    ref = plan.compress_prefill(K, V, ws, want_scores=True)
+    out = plan.compress_prefill_paged(Kp, Vp, table, S, ws, want_scores=True)
+    assert plan.read_status(ws)[0] == 0
+    for key in ("idx", "K_out", "V_out", "scores"):
+        assert torch.equal(ref[key], out[key]), key
+    lay = plan._paged(Kp, table, None)
+    Ko = torch.full_like(ref["K_out"], -3.0)
+    Vo = torch.full_like(ref["V_out"], -3.0)
+    import ctypes
+    rc = plan.lib.lagkv_compress_prefill_paged(plan.handle, binding._ptr(Kp), binding._ptr(Vp), ctypes.byref(lay), S,
+                                               binding._ptr(Ko), binding._ptr(Vo), None, None, binding._ptr(ws),
+                                               ws.numel(), binding._stream(torch.device("cuda", 0)))
+    assert rc == 0 and plan.read_status(ws)[0] == 0
+    assert torch.equal(Ko, ref["K_out"]) and torch.equal(Vo, ref["V_out"])
+
+
 def test_paged_prefill_identity_and_errors(binding, oracle):
     B, H, D, sink, L, k, page = 2, 2, 128, 8, 64, 16, 16
     S = sink + 2 * L - 1                                     # too short: identity
