@@ -75,10 +75,12 @@ def measured_peak():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def kernel_source_hash() -> str:
-    """Hash of the device code: a counter capture stays valid only while this does not change."""
+def kernel_source_hash(files) -> str:
+    """Hash of the device source files a kernel is built from: a counter capture stays valid only
+    while this does not change."""
     h = hashlib.sha256()
-    for f in sorted((ROOT / "paper_2504_04704_b200" / "csrc").glob("*.cuh")):
+    for name in files:
+        f = ROOT / "paper_2504_04704_b200" / "csrc" / name
         h.update(f.name.encode())
         h.update(f.read_bytes())
     return h.hexdigest()[:16]
@@ -86,15 +88,15 @@ def kernel_source_hash() -> str:
 
 def captured_traffic(key: str):
     """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
-    profiles/ncu_traffic.json under ``key`` -- null when there is none, or when the kernels'
-    source has changed since the counters were taken."""
+    profiles/ncu_traffic.json under ``key`` -- null when there is none, or when the kernel's
+    source files have changed since the counters were taken."""
     try:
         rec = json.loads(TRAFFIC_JSON.read_text())[key]
+        if rec["kernel_source_hash"] != kernel_source_hash(rec["source_files"]):
+            return None
+        return rec["traffic_bytes_per_launch"]
     except Exception:
         return None
-    if rec.get("kernel_source_hash") != kernel_source_hash():
-        return None
-    return rec.get("traffic_bytes_per_launch")
 
 
 class ClockSampler:
