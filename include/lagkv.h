@@ -12,14 +12,14 @@
  * rows stay as a sliding window.  The resulting length is Eq. 12.
  *
  * Conventions shared by every entry point
- *   - All cache pointers are DEVICE pointers to 16-bit data (bf16, or fp16 when the plan
- *     says so: "bf16" below stands for the plan's format), 16-byte aligned; scalars and
- *     the config struct are host values.  The library allocates no device memory and
+ *   - All cache pointers are DEVICE pointers to data in the plan's storage format (bf16 by
+ *     default, fp16 or fp8 e4m3 when the plan says so: "bf16" below stands for the plan's
+ *     format), 16-byte aligned; scalars and the config struct are host values.  The library allocates no device memory and
  *     never synchronises the stream, except in lagkv_read_status().
  *   - A cache is addressed as  base + b*stride_b + h*stride_h + s*stride_s + d  (strides
  *     in elements, channel stride 1).  A stride given as 0 means "contiguous
- *     [B, H, S, D]" for the S passed to the call.  Strides must be multiples of 8
- *     elements (16 bytes).
+ *     [B, H, S, D]" for the S passed to the call.  Strides must be multiples of 16 bytes
+ *     (8 elements of a 16-bit format, 16 of fp8).
  *   - "Layers" have no separate dimension: fold them into B (one allocation
  *     [layers*B, H, S, D]) so that one call covers a whole model.
  *   - Every function returning int returns a lagkv_status code (0 = success).
@@ -71,7 +71,15 @@ enum lagkv_variant {
 
 enum lagkv_dtype {
     LAGKV_DTYPE_BF16 = 0, /* the default (a zeroed field)                                */
-    LAGKV_DTYPE_FP16 = 1  /* IEEE binary16 caches                                        */
+    LAGKV_DTYPE_FP16 = 1, /* IEEE binary16 caches                                        */
+    LAGKV_DTYPE_FP8_E4M3 = 2 /* one byte per element: 1 sign, 4 exponent (bias 7), 3 fraction
+                             bits, no infinities, 0x7f / 0xff are NaN (the "e4m3fn" of the
+                             deep-learning frameworks).  The paper names no storage format
+                             and no scale; none is needed: whatever positive per-tensor,
+                             per-head or per-channel scale the caller's quantiser uses, it
+                             cancels in Eq. 9 (the same scale multiplies value, min and max),
+                             so the scores are those of the stored bytes and the kept rows
+                             are copied byte for byte.  head_dim 128 only.                 */
 };
 
 typedef struct {

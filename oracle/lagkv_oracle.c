@@ -8,7 +8,8 @@
  *
  * Every step is written in the order the paper's Methodology lists it, one loop per
  * step, with no blocking, fusion or reordering.  Inputs are 16-bit patterns
- * (uint16_t) in the cache's storage format, bf16 (the default) or IEEE fp16; each is
+ * (uint16_t) in the cache's storage format, bf16 (the default), IEEE fp16, or an fp8 e4m3 byte
+ * zero-extended to 16 bits; each is
  * widened exactly to double before any arithmetic.  The paper does not name a storage
  * format; the method is the same for either.
  *
@@ -42,7 +43,7 @@
 
 enum { LAGKV_ORACLE_LAGKV = 0, LAGKV_ORACLE_LOCALKV = 1, LAGKV_ORACLE_L2NORM = 2 };
 
-enum { LAGKV_ORACLE_BF16 = 0, LAGKV_ORACLE_FP16 = 1 };
+enum { LAGKV_ORACLE_BF16 = 0, LAGKV_ORACLE_FP16 = 1, LAGKV_ORACLE_FP8_E4M3 = 2 };
 
 /* bf16 bit pattern -> double, exact (bf16 is the upper half of an IEEE binary32). */
 static double bf16_to_double(uint16_t bits)
@@ -67,9 +68,26 @@ static double fp16_to_double(uint16_t bits)
     return sign ? -v : v;
 }
 
+/* fp8 "e4m3fn" byte -> double, exact: 1 sign, 4 exponent (bias 7), 3 fraction bits; the format
+ * has no infinities, and exponent 15 with fraction 7 (0x7f, 0xff) is its only NaN.  The byte sits
+ * in the low half of the 16-bit element the oracle's arrays carry (the caller zero-extends). */
+static double fp8_e4m3_to_double(uint16_t bits)
+{
+    int sign = (bits >> 7) & 1, e = (bits >> 3) & 15, frac = bits & 7;
+    double v;
+    if (e == 0)
+        v = ldexp((double)frac, -9);                  /* zero and subnormals: frac/8 * 2^-6 */
+    else if (e == 15 && frac == 7)
+        v = NAN;
+    else
+        v = ldexp(1.0 + (double)frac / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
 /* The storage format of the cache is the only place a value's bits are interpreted. */
 static double decode(uint16_t bits, int storage)
 {
+    if (storage == LAGKV_ORACLE_FP8_E4M3) return fp8_e4m3_to_double(bits);
     return storage == LAGKV_ORACLE_FP16 ? fp16_to_double(bits) : bf16_to_double(bits);
 }
 

@@ -24,7 +24,7 @@ _SRC = _HERE / "lagkv_oracle.c"
 _LIB = _HERE / "liblagkv_oracle.so"
 
 VARIANT_LAGKV, VARIANT_LOCALKV, VARIANT_L2NORM = 0, 1, 2
-STORAGE_BF16, STORAGE_FP16 = 0, 1
+STORAGE_BF16, STORAGE_FP16, STORAGE_FP8_E4M3 = 0, 1, 2
 
 _lib = None
 
@@ -73,9 +73,13 @@ def _ptr(a):
 
 
 def _u16(a) -> np.ndarray:
+    """Bit patterns as the C side takes them: uint16 per element.  fp8 bytes (uint8) are
+    zero-extended: a change of container, not of value."""
     a = np.ascontiguousarray(a)
+    if a.dtype == np.uint8:
+        return a.astype(np.uint16)
     if a.dtype != np.uint16:
-        raise TypeError("K/V must be 16-bit patterns (bf16 or fp16) as uint16")
+        raise TypeError("K/V must be bit patterns: uint16 (bf16, fp16) or uint8 (fp8 e4m3)")
     return a
 
 
@@ -147,6 +151,8 @@ def compress(K, V, static_len: int, L: int, k: int, ddof: int = 1,
         _ptr(K), _ptr(V), B, H, S, D, int(static_len), int(L), int(k), int(ddof), int(variant),
         int(storage), _ptr(idx), _ptr(K_out), _ptr(V_out), _ptr(scores))
     assert got == L_R
+    if storage == STORAGE_FP8_E4M3 and want_rows:     # back to bytes
+        K_out, V_out = K_out.astype(np.uint8), V_out.astype(np.uint8)
     return {"L_R": L_R, "n_c": n_c, "idx": idx, "K_out": K_out, "V_out": V_out, "scores": scores}
 
 
@@ -172,7 +178,7 @@ def compress_append(K_cache, V_cache, seq_len, static_len, L: int, k: int, ddof:
     ``kept[b]`` is ``[H, n_c*k]`` int32 positions (pre-call) of the newly kept rows, or an
     empty array when the sequence was skipped.
     """
-    K_cache, V_cache = _u16(K_cache).copy(), _u16(V_cache).copy()
+    K_cache, V_cache = np.array(K_cache, copy=True), np.array(V_cache, copy=True)
     B = K_cache.shape[0]
     seq_len = np.array(seq_len, dtype=np.int64).copy()
     static_len = np.array(static_len, dtype=np.int64).copy()

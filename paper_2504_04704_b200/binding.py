@@ -149,8 +149,8 @@ def lagkv_keep_for_target(Ls: int, sink: int, lag: int, target_C: float) -> int:
     return int(load_library().lagkv_keep_for_target(int(Ls), int(sink), int(lag), float(target_C)))
 
 
-DTYPE_BF16, DTYPE_FP16 = 0, 1
-_DTYPES = {torch.bfloat16: DTYPE_BF16, torch.float16: DTYPE_FP16}
+DTYPE_BF16, DTYPE_FP16, DTYPE_FP8_E4M3 = 0, 1, 2
+_DTYPES = {torch.bfloat16: DTYPE_BF16, torch.float16: DTYPE_FP16, torch.float8_e4m3fn: DTYPE_FP8_E4M3}
 
 
 class Plan:
@@ -161,7 +161,7 @@ class Plan:
                  variant=VARIANT_LAGKV, strides=(0, 0, 0), device=0, dtype=torch.bfloat16):
         lib = load_library()
         if dtype not in _DTYPES:
-            raise TypeError("dtype must be torch.bfloat16 or torch.float16")
+            raise TypeError("dtype must be torch.bfloat16, torch.float16 or torch.float8_e4m3fn")
         self.dtype = dtype
         self.cfg = lagkv_config(int(B), int(H_kv), int(D), int(sink), int(lag), float(keep_ratio), int(keep_k),
                                 int(std_ddof), int(variant), int(strides[0]), int(strides[1]), int(strides[2]),

@@ -41,6 +41,8 @@ struct KernelTable {
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = ws_paged_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = fp8_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
     }
 };
 const KernelTable& table() {
@@ -62,6 +64,10 @@ int find_kernel(int D, int NW, int TR, int variant, int dtype, bool paged = fals
 }
 
 constexpr int kSmemPerSm = 233472;  // 228 KiB per SM, 1 KiB reserved per resident CTA
+
+// bytes per cache element of a storage format (enum lagkv_dtype)
+int elem_bytes(int dtype) { return dtype == LAGKV_DTYPE_FP8_E4M3 ? 1 : 2; }
+size_t row_bytes(const lagkv_config& c) { return size_t(c.D) * elem_bytes(c.dtype); }
 
 }  // namespace
 
@@ -169,7 +175,7 @@ int make_append_cluster(lagkv_plan_s* pl, int code, int splits, int stages, int 
     const int kidx = find_kernel(pl->cfg.D, code, kAppendPairTileRows, LAGKV_VARIANT_LAGKV, pl->cfg.dtype);
     if (kidx < 0 || pl->cfg.variant != LAGKV_VARIANT_LAGKV) return LAGKV_EUNSUPPORTED;
     const int L = pl->cfg.lag;
-    const size_t rowb = size_t(pl->cfg.D) * 2, per_tile = size_t(kAppendPairTileRows) * rowb + 8;
+    const size_t rowb = row_bytes(pl->cfg), per_tile = size_t(kAppendPairTileRows) * rowb + 8;
     const size_t fixed = kKernels[kidx].smem(stages, L);
     size_t budget = size_t(kSmemPerSm) / size_t(ctas) - 1024;
     if (budget > size_t(pl->max_smem_optin)) budget = size_t(pl->max_smem_optin);
@@ -294,12 +300,13 @@ int resolve_paged(const lagkv_config& c, const lagkv_paged_layout* lay, int64_t 
     long long ss = lay->stride_s ? lay->stride_s : c.D;
     long long sh = lay->stride_h ? lay->stride_h : (long long)ps * ss;
     long long sp = lay->stride_page ? lay->stride_page : (long long)c.H_kv * sh;
-    if (ss < c.D || (ss % 8) || (sh % 8) || (sp % 8) || sh < 0 || sp <= 0) return LAGKV_EINVAL;
-    out->sb = 0;
-    out->sh = sh;
-    out->ss = ss;
+    const int eb = elem_bytes(c.dtype), q = 16 / eb;  // strides are given in elements: multiples of 16 bytes
+    if (ss < c.D || (ss % q) || (sh % q) || (sp % q) || sh < 0 || sp <= 0) return LAGKV_EINVAL;
+    out->sb = 0;  // the kernels count in 16-bit units
+    out->sh = sh * eb / 2;
+    out->ss = ss * eb / 2;
     out->block_table = lay->block_table;
-    out->page_stride = sp;
+    out->page_stride = sp * eb / 2;
     out->max_blocks = lay->max_blocks;
     out->page_shift = 0;
     while ((1 << out->page_shift) < ps) ++out->page_shift;
@@ -330,10 +337,11 @@ int resolve_strides(const lagkv_config& c, int64_t S, Strides* out) {
     long long ss = c.stride_s ? c.stride_s : c.D;
     long long sh = c.stride_h ? c.stride_h : (long long)S * ss;
     long long sb = c.stride_b ? c.stride_b : (long long)c.H_kv * sh;
-    if (ss < c.D || (ss % 8) || (sh % 8) || (sb % 8) || sh < 0 || sb < 0) return LAGKV_EINVAL;
-    out->sb = sb;
-    out->sh = sh;
-    out->ss = ss;
+    const int eb = elem_bytes(c.dtype), q = 16 / eb;  // strides are given in elements: multiples of 16 bytes
+    if (ss < c.D || (ss % q) || (sh % q) || (sb % q) || sh < 0 || sb < 0) return LAGKV_EINVAL;
+    out->sb = sb * eb / 2;  // the kernels count in 16-bit units
+    out->sh = sh * eb / 2;
+    out->ss = ss * eb / 2;
     return LAGKV_OK;
 }
 
@@ -381,9 +389,10 @@ int lagkv_plan(const lagkv_config* cfg, lagkv_plan_t* out) {
     if (cfg->keep_k < 0 || cfg->keep_k > cfg->lag) return LAGKV_EINVAL;
     if (cfg->keep_k == 0 && !(cfg->keep_ratio > 0.0 && cfg->keep_ratio <= 1.0)) return LAGKV_EINVAL;
     if (cfg->stride_b < 0 || cfg->stride_h < 0 || cfg->stride_s < 0) return LAGKV_EINVAL;
-    if (cfg->D <= 0 || (cfg->D % 8) != 0) return LAGKV_EINVAL;
+    if (cfg->dtype != LAGKV_DTYPE_BF16 && cfg->dtype != LAGKV_DTYPE_FP16 && cfg->dtype != LAGKV_DTYPE_FP8_E4M3)
+        return LAGKV_EINVAL;
+    if (cfg->D <= 0 || (cfg->D * elem_bytes(cfg->dtype)) % 16 != 0) return LAGKV_EINVAL;
     if (cfg->variant < LAGKV_VARIANT_LAGKV || cfg->variant > LAGKV_VARIANT_L2NORM) return LAGKV_EINVAL;
-    if (cfg->dtype != LAGKV_DTYPE_BF16 && cfg->dtype != LAGKV_DTYPE_FP16) return LAGKV_EINVAL;
     if (cfg->D != 64 && cfg->D != 96 && cfg->D != 128 && cfg->D != 256) return LAGKV_EUNSUPPORTED;
     if ((long long)cfg->B * cfg->H_kv > (1ll << 30) || 8 * (long long)cfg->H_kv >= kSeqFailed) return LAGKV_EINVAL;
 
@@ -501,13 +510,14 @@ static int prefill_impl(lagkv_plan_t plan, int B, const void* K, const void* V, 
 
     if (rest < 2ll * c.lag) {  // pass skipped: identity
         if (K_out == nullptr && idx_out == nullptr) return LAGKV_OK;
-        const long long total = U * S_in * (c.D / 8);
+        const int vpr = int(row_bytes(c) / 16);
+        const long long total = U * S_in * vpr;
         const int block = 256;
         const long long want = (total + block - 1) / block;
         const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
         lagkv_copy_kernel<<<grid, block, 0, stream>>>(
             static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), cache_layout(st, c.H_kv),
-            int(S_in), c.D / 8, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), idx_out, U);
+            int(S_in), vpr, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), idx_out, U);
         return check_launch();
     }
 
@@ -582,7 +592,7 @@ struct HostSlot {  // byte offsets of one staging slot
     size_t K, V, K_out, V_out, idx, total;
 };
 HostSlot host_slot_layout(const lagkv_plan_s* plan, int64_t S_in, int chunk_B, int64_t L_R) {
-    const size_t units = size_t(chunk_B) * plan->cfg.H_kv, row = size_t(plan->cfg.D) * 2;
+    const size_t units = size_t(chunk_B) * plan->cfg.H_kv, row = row_bytes(plan->cfg);
     HostSlot h;
     h.K = 0;
     h.V = h.K + round256(units * S_in * row);
@@ -637,7 +647,7 @@ int lagkv_compress_prefill_host(lagkv_plan_t plan, const void* K_host, const voi
     bool ok = cudaEventRecord(plan->host_start, user) == cudaSuccess;
     for (int i = 0; i < 3; ++i) ok = ok && cudaStreamWaitEvent(plan->host_stream[i], plan->host_start, 0) == cudaSuccess;
 
-    const size_t units = size_t(chunk_B) * c.H_kv, row = size_t(c.D) * 2;
+    const size_t units = size_t(chunk_B) * c.H_kv, row = row_bytes(c);
     const size_t in_bytes = units * S_in * row, out_bytes = units * L_R * row, idx_bytes = units * L_R * sizeof(int32_t);
     const int chunks = c.B / chunk_B;
     int rc = LAGKV_OK;
@@ -810,13 +820,14 @@ int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, 
     if (n_idx == 0) return LAGKV_OK;
     DeviceGuard guard(c.device);
     const long long U = (long long)c.B * c.H_kv;
-    const long long total = U * n_idx * (c.D / 8);
+    const int vpr = int(row_bytes(c) / 16);
+    const long long total = U * n_idx * vpr;
     const int block = 256;
     const long long want = (total + block - 1) / block;
     const int grid = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
     lagkv_gather_kernel<<<grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), cache_layout(st, c.H_kv), int(S_in),
-        c.D / 8, idx, n_idx, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), U,
+        vpr, idx, n_idx, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), U,
         static_cast<int32_t*>(workspace));
     return check_launch();
 }
@@ -842,7 +853,7 @@ int lagkv_launch_info(lagkv_plan_t plan, int64_t S_in, int32_t info[6]) {
     const long long U = (long long)c.B * c.H_kv;
     const int64_t rest = S_in - c.sink;
     if (rest < 2ll * c.lag) {
-        const long long total = U * S_in * (c.D / 8);
+        const long long total = U * S_in * (long long)(row_bytes(c) / 16);
         const long long want = (total + 255) / 256;
         info[0] = int(want < (long long)plan->sm_count * 16 ? want : (long long)plan->sm_count * 16);
         info[1] = 256;

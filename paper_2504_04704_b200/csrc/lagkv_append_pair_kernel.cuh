@@ -64,8 +64,8 @@ __host__ __device__ inline size_t append_pair_smem_fixed(int stages, int L) {
     size_t s = smem_ring_bytes<G>(stages);              // tile rings (also the staging of the moves)
     s += (size_t(G::NW) * stages + 3) * 8 + 16;         // mbarriers: rings, two for the staged moves, one for the
                                                         // gather (+ those of the resident tiles), padded to 16 bytes
-    s += size_t(G::NW) * 2 * (G::D / 2) * 4;            // min / max partials, one row per warp
-    s += size_t(kAppendMaxSplits) * 2 * (G::D / 2) * 4; // min / max rows of the row splits
+    s += size_t(G::NW) * 2 * G::STAT * 4;            // min / max partials, one row per warp
+    s += size_t(kAppendMaxSplits) * 2 * G::STAT * 4; // min / max rows of the row splits
     s += sizeof(SelScratch);
     s = (s + 15) & ~size_t(15);
     s += size_t(2) * ((L + 3) & ~3) * 4;                // sigma of K and of V
@@ -80,8 +80,8 @@ __host__ __device__ inline size_t append_pair_smem_fixed(int stages, int L) {
 template <class G, class Src>
 __device__ bool move_rows_staged(uint16_t* X, long long ss, int dst_row0, int total, Src src, bool src_contiguous,
                                  uint32_t stage0, int R, uint32_t bar0, int& chunk0, int lane) {
-    constexpr uint32_t ROWB = G::D * 2;
-    const bool contiguous = ss == G::D;
+    constexpr uint32_t ROWB = G::ROWB;
+    const bool contiguous = ss == G::ROW16;
     const int nchunks = (total + R - 1) / R;
     auto load = [&](int c) {
         const int j0 = c * R, nr = min(R, total - j0), g = chunk0 + c;
@@ -131,8 +131,8 @@ template <class G>
 __global__ void __launch_bounds__(G::NT, (G::NW <= 4 ? 2 : 1)) lagkv_append_pair_kernel(const Params P) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    constexpr uint32_t ROWB = G::D * 2;
-    constexpr int STAT = G::D / 2;      // packed words per min (or max) row
+    constexpr uint32_t ROWB = G::ROWB;
+    constexpr int STAT = G::STAT;      // packed words per min (or max) row
     const int NS = P.stages;
     const int res_tiles = P.res_tiles;  // room for that many resident tiles (the same in every CTA)
     unsigned char* ring = sm;
@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW <= 4 ? 2 : 1)) lagkv_append_pair
     const int cg = lane % G::LPR, rl = lane / G::LPR;
     const int L = P.L, k = P.k;
     const int ntiles = (L + G::TR - 1) / G::TR;
-    const bool contiguous = (P.ss == G::D);
+    const bool contiguous = (P.ss == G::ROW16);
     const uint32_t rank = cluster_ctarank(), CS = cluster_nctarank();
     const int tensor = int(rank & 1u);           // 0: this CTA handles K, 1: V
     const int RS = int(CS >> 1), h = int(rank >> 1);  // row splits per tensor, this CTA's split
@@ -238,10 +238,10 @@ __global__ void __launch_bounds__(G::NT, (G::NW <= 4 ? 2 : 1)) lagkv_append_pair
     int cslot = 0;
     uint32_t cparity = 0;
     const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
-    f32x2 a2[G::NWORD], b2[G::NWORD];
-    uint32_t mn[G::NWORD], mx[G::NWORD];
+    f32x2 a2[G::NPW], b2[G::NPW];
+    uint32_t mn[G::NPW], mx[G::NPW];
 #pragma unroll
-    for (int j = 0; j < G::NWORD; ++j) {
+    for (int j = 0; j < G::NPW; ++j) {
         a2[j] = b2[j] = 0ull;
         mn[j] = G::E::kPosInf2;
         mx[j] = G::E::kNegInf2;
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW <= 4 ? 2 : 1)) lagkv_append_pair
         ring_advance();
     }
 #pragma unroll
-    for (int j = 0; j < G::NWORD; ++j) {
+    for (int j = 0; j < G::NPW; ++j) {
 #pragma unroll
         for (int o = G::LPR; o < 32; o <<= 1) {
             mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
@@ -296,14 +296,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW <= 4 ? 2 : 1)) lagkv_append_pair
         }
     }
     if (rl == 0) {
-        uint32_t* st = stats + warp * 2 * STAT;
-#pragma unroll
-        for (int v = 0; v < G::V; ++v)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                st[(v * G::LPR + cg) * 4 + c] = mn[v * 4 + c];
-                st[STAT + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
-            }
+        store_stats_row<G>(stats + warp * 2 * STAT, mn, mx, cg);
     }
     __syncthreads();
     cluster_wait();  // every CTA of the cluster is running: its shared memory may be written

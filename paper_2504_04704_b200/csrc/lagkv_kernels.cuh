@@ -215,6 +215,9 @@ template <int DT>
 struct Elem;
 template <>
 struct Elem<0> {  // bf16: the upper half of an IEEE binary32
+    static constexpr int EB = 2;  // bytes per element
+    static constexpr int PW = 1;  // packed pairs per 32-bit word of cache data
+    static __device__ __forceinline__ void expand(uint32_t w, uint32_t (&p)[1]) { p[0] = w; }
     static constexpr uint32_t kPosInf2 = 0x7f807f80u, kNegInf2 = 0xff80ff80u;
     static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
         uint32_t r;
@@ -231,6 +234,9 @@ struct Elem<0> {  // bf16: the upper half of an IEEE binary32
 };
 template <>
 struct Elem<1> {  // fp16: IEEE binary16
+    static constexpr int EB = 2;
+    static constexpr int PW = 1;
+    static __device__ __forceinline__ void expand(uint32_t w, uint32_t (&p)[1]) { p[0] = w; }
     static constexpr uint32_t kPosInf2 = 0x7c007c00u, kNegInf2 = 0xfc00fc00u;
     static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
         uint32_t r;
@@ -251,6 +257,20 @@ struct Elem<1> {  // fp16: IEEE binary16
         float f;
         asm("{ .reg .b16 l, h; mov.b32 {l, h}, %1; cvt.f32.f16 %0, h; }" : "=f"(f) : "r"(w));
         return f;
+    }
+};
+// fp8 (e4m3, finite-only: the "fn" flavour, no infinities, 0x7f / 0xff are NaN): four values per
+// word.  Every e4m3 value is a binary16 value, so a word is first expanded exactly into two packed
+// fp16 pairs (one conversion instruction each) and from there on treated like fp16 data: packed
+// min / max, exact widening to fp32.
+template <>
+struct Elem<2> : Elem<1> {
+    static constexpr int EB = 1;
+    static constexpr int PW = 2;
+    static __device__ __forceinline__ void expand(uint32_t w, uint32_t (&p)[2]) {
+        asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.rn.f16x2.e4m3x2 %0, l; cvt.rn.f16x2.e4m3x2 %1, h; }"
+            : "=r"(p[0]), "=r"(p[1])
+            : "r"(w));
     }
 };
 // two packed 16-bit values in one word -> two fp32 (exact)
@@ -308,18 +328,23 @@ template <int D_, int V_, int NW_, int TR_, int DT_ = 0>
 struct Geo {
     using E = Elem<DT_>;                   // storage format of the cache elements
     static constexpr int DT = DT_;
-    static constexpr int D = D_;           // head_dim
+    static constexpr int D = D_;           // head_dim (channels per row)
     static constexpr int V = V_;           // 16-byte vectors per thread per row
     static constexpr int NW = NW_;         // warps per CTA (even: K warps, odd: V warps)
     static constexpr int TR = TR_;         // rows per staged tile
     static constexpr int NT = NW * 32;
     static constexpr int WT = NW / 2;      // warps per tensor
-    static constexpr int VPR = D / 8;      // 16-byte vectors per row
+    static constexpr int ROWB = D * E::EB; // bytes per row
+    static constexpr int ROW16 = ROWB / 2; // row length in the 16-bit units the cache pointers count in
+    static constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
     static constexpr int LPR = VPR / V;    // lanes per row
     static constexpr int RPL = 32 / LPR;   // rows per warp-wide load
     static constexpr int NV = TR / RPL;    // row partials per thread per tile
-    static constexpr int NWORD = 4 * V;    // packed bf16x2 words per thread per row
-    static constexpr int TILE_BYTES = TR * D * 2;
+    static constexpr int NWORD = 4 * V;    // 32-bit words of cache data per thread per row
+    static constexpr int PW = E::PW;       // packed pairs of channels per such word (2 for fp8)
+    static constexpr int NPW = NWORD * PW; // packed pairs per thread per row: min / max / coefficient registers
+    static constexpr int STAT = D / 2;     // packed pairs per min (or max) row of a tensor
+    static constexpr int TILE_BYTES = TR * ROWB;
     static_assert(LPR * V == VPR && RPL * LPR == 32 && NV * RPL == TR, "bad geometry");
     static_assert(NV >= 1 && NV <= LPR, "tile too tall for the transposed reduction");
     static_assert(NW >= 2 && NW <= kMaxWarps && (NW % 2) == 0, "bad warp count");
@@ -346,7 +371,7 @@ template <class G>
 __host__ __device__ inline size_t smem_total_bytes(int stages, int L) {
     size_t s = smem_ring_bytes<G>(stages);         // tile rings
     s += size_t(G::NW) * stages * 8 + 16;          // mbarriers: the rings', and two for the append move
-    s += size_t(2) * G::WT * 2 * (G::D / 2) * 4;   // per-warp min/max partials
+    s += size_t(2) * G::WT * 2 * G::STAT * 4;   // per-warp min/max partials
     s += sizeof(SelScratch);
     s = (s + 15) & ~size_t(15);
     s += size_t(2) * ((L + 3) & ~3) * 4;           // sigma / score / kept arrays
@@ -380,8 +405,8 @@ __device__ __forceinline__ void transposed_reduce(float (&v)[NV], int cg) {
 // writes sigma (Std. of Eq. 10) for every valid row.
 template <class G, bool SCORE, bool FULL, bool STATS = true>
 __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int nrows,
-                                             const f32x2 (&a2)[G::NWORD], const f32x2 (&b2)[G::NWORD],
-                                             uint32_t (&mn)[G::NWORD], uint32_t (&mx)[G::NWORD],
+                                             const f32x2 (&a2)[G::NPW], const f32x2 (&b2)[G::NPW],
+                                             uint32_t (&mn)[G::NPW], uint32_t (&mx)[G::NPW],
                                              float* __restrict__ sig_out, float inv_D, float inv_Dm,
                                              int lane) {
     const int cg = lane % G::LPR, rl = lane / G::LPR;
@@ -397,15 +422,20 @@ __device__ __forceinline__ void process_tile(const uint4* __restrict__ tile, int
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const int j = v * 4 + c;
-                if (STATS && valid) {
-                    mn[j] = G::E::min2(mn[j], w[c]);
-                    mx[j] = G::E::max2(mx[j], w[c]);
-                }
-                if (SCORE) {
-                    const f32x2 y = fma2(widen2<typename G::E>(w[c]), a2[j], b2[j]);  // Eq. 9 (centred)
-                    s1 = add2(s1, y);
-                    s2 = fma2(y, y, s2);
+                uint32_t pw[G::PW];
+                G::E::expand(w[c], pw);
+#pragma unroll
+                for (int q = 0; q < G::PW; ++q) {
+                    const int j = (v * 4 + c) * G::PW + q;
+                    if (STATS && valid) {
+                        mn[j] = G::E::min2(mn[j], pw[q]);
+                        mx[j] = G::E::max2(mx[j], pw[q]);
+                    }
+                    if (SCORE) {
+                        const f32x2 y = fma2(widen2<typename G::E>(pw[q]), a2[j], b2[j]);  // Eq. 9 (centred)
+                        s1 = add2(s1, y);
+                        s2 = fma2(y, y, s2);
+                    }
                 }
             }
         }
@@ -447,8 +477,13 @@ __device__ __forceinline__ void process_tile_l2(const uint4* __restrict__ tile, 
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const f32x2 z = widen2<typename G::E>(w[c]);
-                s2 = fma2(z, z, s2);
+                uint32_t pw[G::PW];
+                G::E::expand(w[c], pw);
+#pragma unroll
+                for (int q = 0; q < G::PW; ++q) {
+                    const f32x2 z = widen2<typename G::E>(pw[q]);
+                    s2 = fma2(z, z, s2);
+                }
             }
         }
         float lo, hi;
@@ -461,6 +496,20 @@ __device__ __forceinline__ void process_tile_l2(const uint4* __restrict__ tile, 
     if ((cg % DUP) == 0 && (FULL || row < nrows)) norm_out[row] = sqrtf(p2[0]);
 }
 
+// This lane's packed min / max pairs -> its places in a [mn | mx] row of shared memory (STAT words
+// each; the lane owns 4 * PW consecutive words per 16-byte vector of cache data it reads).
+template <class G>
+__device__ __forceinline__ void store_stats_row(uint32_t* st, const uint32_t (&mn)[G::NPW], const uint32_t (&mx)[G::NPW],
+                                                int cg) {
+#pragma unroll
+    for (int v = 0; v < G::V; ++v)
+#pragma unroll
+        for (int c = 0; c < 4 * G::PW; ++c) {
+            st[(v * G::LPR + cg) * 4 * G::PW + c] = mn[v * 4 * G::PW + c];
+            st[G::STAT + (v * G::LPR + cg) * 4 * G::PW + c] = mx[v * 4 * G::PW + c];
+        }
+}
+
 // ------------------------------------------------------------------ coefficients of Eq. 9
 // Combine the per-warp min / max partials of one tensor (nw rows of [mn | mx], STAT words
 // each, packed bf16x2) and turn them into y = a * z + b for this lane's channels:
@@ -469,20 +518,21 @@ __device__ __forceinline__ void process_tile_l2(const uint4* __restrict__ tile, 
 // had zero range.  The reciprocal is the hardware approximation (1 ulp), the same in every
 // kernel, so scores do not depend on which kernel ran.
 template <class G>
-__device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw, int cg, f32x2 (&a2)[G::NWORD],
-                                                 f32x2 (&b2)[G::NWORD]) {
-    constexpr int STAT = G::D / 2;
-    uint32_t fmn[G::NWORD], fmx[G::NWORD];
+__device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw, int cg, f32x2 (&a2)[G::NPW],
+                                                 f32x2 (&b2)[G::NPW]) {
+    constexpr int STAT = G::STAT;
+    uint32_t fmn[G::NPW], fmx[G::NPW];
 #pragma unroll
-    for (int j = 0; j < G::NWORD; ++j) {
+    for (int j = 0; j < G::NPW; ++j) {
         fmn[j] = G::E::kPosInf2;
         fmx[j] = G::E::kNegInf2;
     }
     for (int w = 0; w < nw; ++w) {
         const uint4* st = reinterpret_cast<const uint4*>(stats_t + w * 2 * STAT);
 #pragma unroll
-        for (int v = 0; v < G::V; ++v) {
-            const uint4 lo = st[v * G::LPR + cg], hi = st[STAT / 4 + v * G::LPR + cg];
+        for (int v = 0; v < G::V * G::PW; ++v) {  // this lane's pairs: 4 * PW per vector, four to a 16-byte load
+            const int i = (v / G::PW * G::LPR + cg) * G::PW + v % G::PW;
+            const uint4 lo = st[i], hi = st[STAT / 4 + i];
             fmn[v * 4 + 0] = G::E::min2(fmn[v * 4 + 0], lo.x);
             fmn[v * 4 + 1] = G::E::min2(fmn[v * 4 + 1], lo.y);
             fmn[v * 4 + 2] = G::E::min2(fmn[v * 4 + 2], lo.z);
@@ -495,7 +545,7 @@ __device__ __forceinline__ int make_coefficients(const uint32_t* stats_t, int nw
     }
     int zero_range = 0;
 #pragma unroll
-    for (int j = 0; j < G::NWORD; ++j) {
+    for (int j = 0; j < G::NPW; ++j) {
         const float lo0 = G::E::lo(fmn[j]), lo1 = G::E::hi(fmn[j]);
         const float hi0 = G::E::lo(fmx[j]), hi1 = G::E::hi(fmx[j]);
         const float r0 = hi0 - lo0, r1 = hi1 - lo1;
@@ -966,9 +1016,9 @@ template <class G>
 __device__ bool move_rows_bulk(uint16_t* K, uint16_t* V, const RowMap& m, int dst_row0, int total, int n_kept,
                                const int32_t* kept_pos, int win_src0, uint32_t stage0, int R,
                                uint32_t bar0, int lane) {
-    constexpr uint32_t ROWB = G::D * 2;
+    constexpr uint32_t ROWB = G::ROWB;
     const uint32_t stage_bytes = 2u * uint32_t(R) * ROWB;
-    const bool dense = m.ss == G::D;
+    const bool dense = m.ss == G::ROW16;
     const int nchunks = (total + R - 1) / R;
     auto load = [&](int c) {
         const int j0 = c * R, nr = min(R, total - j0);
@@ -1028,7 +1078,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     uint64_t* bars = reinterpret_cast<uint64_t*>(ring + smem_ring_bytes<G>(NS));
     uint64_t* move_bars = bars + G::NW * NS;  // two more for the in-place move of the append pass
     uint32_t* stats = reinterpret_cast<uint32_t*>(move_bars + 2);  // [2][WT][2][D/2]
-    SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * G::WT * 2 * (G::D / 2));
+    SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * G::WT * 2 * G::STAT);
     float* sg = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
     const int Lp = (P.L + 3) & ~3;
     float* sg0 = sg;
@@ -1039,7 +1089,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     const int cg = lane % G::LPR, rl = lane / G::LPR;
     const int L = P.L, k = P.k;
     const int ntiles = (L + G::TR - 1) / G::TR;
-    const bool contiguous = (P.ss == G::D);
+    const bool contiguous = (P.ss == G::ROW16);
 
     // Slot j of a unit.  LagKV (Eq. 7-9): partitions n-1 ... 0, each scored with the statistics
     // of the slot before it.  LocalKV (Eq. 14, Eq. 15): partitions n-2 ... 0, each visited twice
@@ -1122,9 +1172,9 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         const uint32_t bar = bar_w + 8 * pslot;
         if (lane == 0) {
             fence_proxy_async();
-            mbar_arrive_expect_tx(bar, uint32_t(rows) * G::D * 2);
+            mbar_arrive_expect_tx(bar, uint32_t(rows) * G::ROWB);
         }
-        fetch_rows(tbase, pmap, row0, rows, dst, bar, G::D * 2, contiguous, lane);
+        fetch_rows(tbase, pmap, row0, rows, dst, bar, G::ROWB, contiguous, lane);
         pt += G::WT;
         if (pt >= ntiles) {
             pt = wj;
@@ -1139,9 +1189,9 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
     bool timed_out = false, aborted = false;
     const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
 
-    f32x2 a2[G::NWORD], b2[G::NWORD];
+    f32x2 a2[G::NPW], b2[G::NPW];
 #pragma unroll
-    for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
+    for (int j = 0; j < G::NPW; ++j) a2[j] = b2[j] = 0ull;
     bool have_ref = false;
 
     for (long long s = s_lo; s < s_hi; ++s) {
@@ -1149,9 +1199,9 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         const bool first_of_unit = sj == 0, last_of_unit = sj == spu - 1;
         const bool score = scored(sj) && s >= s_first && (have_ref || !needs_prev(sj));
 
-        uint32_t mn[G::NWORD], mx[G::NWORD];
+        uint32_t mn[G::NPW], mx[G::NPW];
 #pragma unroll
-        for (int j = 0; j < G::NWORD; ++j) {
+        for (int j = 0; j < G::NPW; ++j) {
             mn[j] = G::E::kPosInf2;  // +inf, +inf
             mx[j] = G::E::kNegInf2;  // -inf, -inf
         }
@@ -1192,7 +1242,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
 
         // ---- this partition's min / max (Eq. 7, Eq. 8): lanes sharing channels, then warps
 #pragma unroll
-        for (int j = 0; j < G::NWORD; ++j) {
+        for (int j = 0; j < G::NPW; ++j) {
 #pragma unroll
             for (int o = G::LPR; o < 32; o <<= 1) {
                 mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
@@ -1200,14 +1250,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
             }
         }
         if (rl == 0) {
-            uint32_t* st = stats + ((tensor * G::WT + wj) * 2) * (G::D / 2);
-#pragma unroll
-            for (int v = 0; v < G::V; ++v)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    st[(v * G::LPR + cg) * 4 + c] = mn[v * 4 + c];
-                    st[(G::D / 2) + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
-                }
+            store_stats_row<G>(stats + ((tensor * G::WT + wj) * 2) * G::STAT, mn, mx, cg);
         }
         __syncthreads();
         aborted = *reinterpret_cast<volatile int*>(&sc.abort) != 0;
@@ -1226,8 +1269,8 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
             const int* kept = reinterpret_cast<const int*>(sg1);
             if (P.mode == MODE_PREFILL) {
                 emit_kept<G::NT, G::VPR>(P.K, P.V, make_rowmap(P, u),
-                                         P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr,
-                                         P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr,
+                                         P.K_out ? P.K_out + (long long)u * P.L_R * G::ROW16 : nullptr,
+                                         P.V_out ? P.V_out + (long long)u * P.L_R * G::ROW16 : nullptr,
                                          stat_rows + p * L, stat_rows + p * k, kept, k,
                                          P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr, tid);
             } else {
@@ -1238,7 +1281,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
 
         // ---- coefficients for the next (lower) partition from this one's statistics
         {
-            const int zero_range = make_coefficients<G>(stats + (tensor * G::WT) * 2 * (G::D / 2), G::WT, cg, a2, b2);
+            const int zero_range = make_coefficients<G>(stats + (tensor * G::WT) * 2 * G::STAT, G::WT, cg, a2, b2);
             if (zero_range != 0 && wj == 0 && rl == 0 && !l2norm && P.status != nullptr)
                 atomicAdd(P.status + 2, zero_range);
             have_ref = true;
@@ -1247,8 +1290,8 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         // ---- rows copied verbatim (prefill): window with a unit's first slot, sink with its last
         if (P.mode == MODE_PREFILL && s >= s_first) {
             const RowMap um = make_rowmap(P, u);
-            uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
-            uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
+            uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::ROW16 : nullptr;
+            uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::ROW16 : nullptr;
             int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
             if (first_of_unit)
                 copy_rows<G::NT, G::VPR>(P.K, P.V, um, ok, ov, stat_rows + (n - 1) * L, stat_rows + (n - 1) * k,
@@ -1267,7 +1310,7 @@ __global__ void __launch_bounds__(G::NT, (G::NW == 2 ? 6 : 1)) lagkv_stream_kern
         const int n_c = n - 1;
         const int32_t* kp = P.kept_pos + (long long)u * P.max_chunks * k;
         if (!aborted && k < L && warp == 0) {  // kept rows, then the window, as one ascending sequence of rows
-            const int R = int(smem_ring_bytes<G>(NS) / (4 * G::D * 2));
+            const int R = int(smem_ring_bytes<G>(NS) / (4 * G::ROWB));
             if (!move_rows_bulk<G>(ck, cv, make_rowmap(P, u), stat_rows, n_c * k + L + rem, n_c * k, kp,
                                    stat_rows + n_c * L - n_c * k, smem_u32(ring), R, smem_u32(move_bars), lane)) {
                 timed_out = true;

@@ -30,7 +30,7 @@ __host__ __device__ inline size_t pair_smem_total_bytes(int stages, int L) {
     const size_t Lp = (L + 3) & ~3;
     size_t s = smem_ring_bytes<G>(stages);             // tile rings
     s += (size_t(G::NW) * stages + 4 * kPairs) * 8;    // mbarriers: rings, full[2] / empty[2] per pair
-    s += size_t(G::NW) * 2 * (G::D / 2) * 4;           // own min / max row of every streaming warp
+    s += size_t(G::NW) * 2 * G::STAT * 4;           // own min / max row of every streaming warp
     s += size_t(kPairs) * 2 * 2 * Lp * 4;              // sigma [pair][2 buffers][K, V]
     s += size_t(kPairs) * Lp * 4;                      // kept indices [pair]
     s += size_t(kPairs) * 4;                           // give-up flag [pair]
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const int NS = P.stages;
-    constexpr int STAT_WORDS = G::D / 2;  // packed bf16x2 words per min (or max) row
+    constexpr int STAT_WORDS = G::STAT;  // packed bf16x2 words per min (or max) row
     unsigned char* ring = sm;
     uint64_t* bars = reinterpret_cast<uint64_t*>(ring + smem_ring_bytes<G>(NS));
     uint64_t* xbars = bars + G::NW * NS;  // per pair: full[2], empty[2]
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = P.L, k = P.k, n = P.n, sink = P.sink;
     const int ntiles = (L + G::TR - 1) / G::TR;
-    const bool contiguous = (P.ss == G::D);
+    const bool contiguous = (P.ss == G::ROW16);
     const bool streamer = warp < G::NW;
     const int pair = streamer ? (warp >> 1) : (warp - G::NW);
 
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             const uint16_t* src = pbase + (long long)row0 * P.ss;
             const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
             const uint32_t bar = bar_w + 8 * pslot;
-            const uint32_t bytes = uint32_t(rows) * G::D * 2;
+            const uint32_t bytes = uint32_t(rows) * G::ROWB;
             if (lane == 0) {
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar, bytes);
@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             } else {
                 __syncwarp();
                 for (int r = lane; r < rows; r += 32)
-                    bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+                    bulk_g2s(dst + uint32_t(r) * G::ROWB, src + (long long)r * P.ss, G::ROWB, bar);
             }
             if (++pt == ntiles) {  // next slot: the partition below, or the top of the next unit
                 pt = 0;
@@ -253,9 +253,9 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
         int cslot = 0;
         uint32_t cparity = 0;
         const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
-        f32x2 a2[G::NWORD], b2[G::NWORD];
+        f32x2 a2[G::NPW], b2[G::NPW];
 #pragma unroll
-        for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
+        for (int j = 0; j < G::NPW; ++j) a2[j] = b2[j] = 0ull;
 
         int p = n - 1 - int(s_lo % n);
         for (long long s = s_lo; s < s_hi; ++s, p = (p == 0 ? n - 1 : p - 1)) {
@@ -264,9 +264,9 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             // the epilogue warp must have released this sigma buffer (slot i - 2)
             if (i >= 2 && !dead && !mbar_wait_bounded(empty_bar + 8 * buf, uint32_t((i >> 1) - 1) & 1u)) give_up();
 
-            uint32_t mn[G::NWORD], mx[G::NWORD];
+            uint32_t mn[G::NPW], mx[G::NPW];
 #pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
+            for (int j = 0; j < G::NPW; ++j) {
                 mn[j] = G::E::kPosInf2;  // +inf, +inf
                 mx[j] = G::E::kNegInf2;  // -inf, -inf
             }
@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             // ---- this partition's min / max (Eq. 7, Eq. 8) across the lanes sharing channels,
             //      then the coefficients for the next (lower) partition
 #pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
+            for (int j = 0; j < G::NPW; ++j) {
 #pragma unroll
                 for (int o = G::LPR; o < 32; o <<= 1) {
                     mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
@@ -310,13 +310,7 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
                 }
             }
             if (rl == 0) {
-                uint4* st = reinterpret_cast<uint4*>(stats_w);
-#pragma unroll
-                for (int v = 0; v < G::V; ++v) {
-                    st[v * G::LPR + cg] = make_uint4(mn[v * 4], mn[v * 4 + 1], mn[v * 4 + 2], mn[v * 4 + 3]);
-                    st[STAT_WORDS / 4 + v * G::LPR + cg] =
-                        make_uint4(mx[v * 4], mx[v * 4 + 1], mx[v * 4 + 2], mx[v * 4 + 3]);
-                }
+                store_stats_row<G>(stats_w, mn, mx, cg);
             }
             __syncwarp();
             const int zero_range = make_coefficients<G>(stats_w, 1, cg, a2, b2);
@@ -340,8 +334,8 @@ __global__ void __launch_bounds__(G::NT + kPairs * 32, 1) lagkv_pair_kernel(cons
             if (!dead && __shfl_sync(0xffffffffu, gave_up[pair], 0) != 0) dead = true;
             const uint32_t ebar = empty_bar + 8 * buf;
             const RowMap um = make_rowmap(P, u);
-            uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::D : nullptr;
-            uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::D : nullptr;
+            uint16_t* ok = P.K_out ? P.K_out + (long long)u * P.L_R * G::ROW16 : nullptr;
+            uint16_t* ov = P.V_out ? P.V_out + (long long)u * P.L_R * G::ROW16 : nullptr;
             int32_t* oi = P.idx_out ? P.idx_out + (long long)u * P.L_R : nullptr;
             if (score && !dead) {
                 const float* sg0 = sg_pair + (buf * 2) * Lp;

@@ -52,11 +52,12 @@ constexpr int kAppendPairTileRows = 16;
 /* the two shapes the planner uses for appends, also for the LocalKV and L2-norm variants */
 #define LAGKV_VARIANT_ENTRIES(D, V) \
     LAGKV_ENTRY1(D, V, 4, 32, 1), LAGKV_ENTRY1(D, V, 4, 32, 2), LAGKV_ENTRY1(D, V, 2, 16, 1), LAGKV_ENTRY1(D, V, 2, 16, 2)
-/* fp16 caches: the planner's default shapes, every variant */
-#define LAGKV_FP16_ENTRIES(D, V) \
-    LAGKV_ENTRY2(D, V, 8, 32, 0, 1), LAGKV_ENTRY2(D, V, 4, 32, 0, 1), LAGKV_ENTRY2(D, V, 2, 16, 0, 1), \
-    LAGKV_ENTRY2(D, V, 4, 32, 1, 1), LAGKV_ENTRY2(D, V, 4, 32, 2, 1), LAGKV_ENTRY2(D, V, 2, 16, 1, 1), \
-    LAGKV_ENTRY2(D, V, 2, 16, 2, 1)
+/* fp16 (or another format's) caches: the planner's default shapes, every variant */
+#define LAGKV_FP16_ENTRIES_DT(D, V, DT) \
+    LAGKV_ENTRY2(D, V, 8, 32, 0, DT), LAGKV_ENTRY2(D, V, 4, 32, 0, DT), LAGKV_ENTRY2(D, V, 2, 16, 0, DT), \
+    LAGKV_ENTRY2(D, V, 4, 32, 1, DT), LAGKV_ENTRY2(D, V, 4, 32, 2, DT), LAGKV_ENTRY2(D, V, 2, 16, 1, DT), \
+    LAGKV_ENTRY2(D, V, 2, 16, 2, DT)
+#define LAGKV_FP16_ENTRIES(D, V) LAGKV_FP16_ENTRIES_DT(D, V, 1)
 #define LAGKV_WS_ENTRY2(D, V, NWS, TR, VAR, DT) \
     { D, NWS + kWsEpiWarps, TR, VAR, DT, true, (NWS + kWsEpiWarps) * 32, \
       &lagkv_ws_kernel<Geo<D, V, NWS, TR, DT>, VAR>, &ws_smem_total_bytes<Geo<D, V, NWS, TR, DT>> }
@@ -68,5 +69,6 @@ constexpr int kAppendPairTileRows = 16;
     { D, NWS + kWsEpiWarps, TR, 0, DT, true, (NWS + kWsEpiWarps) * 32, \
       &lagkv_ws_kernel<Geo<D, V, NWS, TR, DT>, 0, true>, &ws_smem_total_bytes<Geo<D, V, NWS, TR, DT>>, true }
 int ws_paged_kernels(const KernelEntry** table);      // lagkv_ws_kernel reading paged caches
+int fp8_kernels(const KernelEntry** table);           // every family for fp8 (e4m3) caches, head_dim 128
 
 }  // namespace lagkv

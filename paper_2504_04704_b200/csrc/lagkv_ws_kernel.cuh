@@ -40,9 +40,9 @@ constexpr int kBarSelect = 3;       // named barrier 3: the select warps
 template <class G>
 __host__ __device__ inline size_t ws_smem_total_bytes(int stages, int L) {
     size_t s = smem_ring_bytes<G>(stages);                  // tile rings
-    s += size_t(2) * 2 * kWsCopyRows * G::D * 2;            // copy staging [2 stages][K, V]
+    s += size_t(2) * 2 * kWsCopyRows * G::ROWB;            // copy staging [2 stages][K, V]
     s += (size_t(G::NW) * stages + 6) * 8;                  // mbarriers
-    s += size_t(2) * 2 * G::WT * 2 * (G::D / 2) * 4;        // min/max partials [2][K,V][WT][mn,mx]
+    s += size_t(2) * 2 * G::WT * 2 * G::STAT * 4;        // min/max partials [2][K,V][WT][mn,mx]
     s += sizeof(SelScratch);
     s = (s + 15) & ~size_t(15);
     s += size_t(2) * 2 * ((L + 3) & ~3) * 4;                // sigma [2 buffers][K, V]
@@ -60,13 +60,13 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const int NS = P.stages;
-    constexpr int CHUNK_BYTES = kWsCopyRows * G::D * 2;     // one tensor, one staged chunk
+    constexpr int CHUNK_BYTES = kWsCopyRows * G::ROWB;     // one tensor, one staged chunk
     unsigned char* ring = sm;
     unsigned char* stage = ring + smem_ring_bytes<G>(NS);
     uint64_t* bars = reinterpret_cast<uint64_t*>(stage + 4 * CHUNK_BYTES);
     uint64_t* xbars = bars + G::NW * NS;                    // full[2], empty[2], copy[2]
     uint32_t* stats = reinterpret_cast<uint32_t*>(xbars + 6);
-    constexpr int STAT_WORDS = G::D / 2;                    // packed bf16x2 words per min (or max) row
+    constexpr int STAT_WORDS = G::STAT;                    // packed bf16x2 words per min (or max) row
     SelScratch& sc = *reinterpret_cast<SelScratch*>(stats + 2 * 2 * G::WT * 2 * STAT_WORDS);
     float* sgbase = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(&sc + 1) + 15) & ~uintptr_t(15));
     const int Lp = (P.L + 3) & ~3;
@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = P.L, k = P.k, n = P.n, sink = P.sink;
     const int ntiles = (L + G::TR - 1) / G::TR;
-    const bool contiguous = (P.ss == G::D);
+    const bool contiguous = (P.ss == G::ROW16);
 
     // slots [s_first, s_hi) belong to this CTA; a range that starts inside a unit first
     // re-reads the partition above it (statistics only)
@@ -151,13 +151,13 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             const int rows = min(G::TR, L - pt * G::TR);
             const uint32_t dst = ring_w + uint32_t(pslot) * G::TILE_BYTES;
             const uint32_t bar = bar_w + 8 * pslot;
-            const uint32_t bytes = uint32_t(rows) * G::D * 2;
+            const uint32_t bytes = uint32_t(rows) * G::ROWB;
             if (lane == 0) {
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar, bytes);
             }
             if (PAGED) {
-                fetch_rows(tbase, pmap, row0, rows, dst, bar, G::D * 2, contiguous, lane);
+                fetch_rows(tbase, pmap, row0, rows, dst, bar, G::ROWB, contiguous, lane);
             } else {
                 const uint16_t* src = pbase + (long long)row0 * P.ss;
                 if (contiguous) {
@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 } else {
                     __syncwarp();
                     for (int r = lane; r < rows; r += 32)
-                        bulk_g2s(dst + uint32_t(r) * G::D * 2, src + (long long)r * P.ss, G::D * 2, bar);
+                        bulk_g2s(dst + uint32_t(r) * G::ROWB, src + (long long)r * P.ss, G::ROWB, bar);
                 }
             }
             pt += WTE;
@@ -186,9 +186,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
         int cslot = 0;
         uint32_t cparity = 0;
         const float inv_D = 1.0f / float(G::D), inv_Dm = 1.0f / float(G::D - P.ddof);
-        f32x2 a2[G::NWORD], b2[G::NWORD];
+        f32x2 a2[G::NPW], b2[G::NPW];
 #pragma unroll
-        for (int j = 0; j < G::NWORD; ++j) a2[j] = b2[j] = 0ull;
+        for (int j = 0; j < G::NPW; ++j) a2[j] = b2[j] = 0ull;
 
         int cj = int(s_lo % spu);
         for (long long s = s_lo; s < s_hi; ++s, cj = (cj + 1 == spu ? 0 : cj + 1)) {
@@ -201,9 +201,9 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 raise_abort();
             }
 
-            uint32_t mn[G::NWORD], mx[G::NWORD];
+            uint32_t mn[G::NPW], mx[G::NPW];
 #pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
+            for (int j = 0; j < G::NPW; ++j) {
                 mn[j] = G::E::kPosInf2;  // +inf, +inf
                 mx[j] = G::E::kNegInf2;  // -inf, -inf
             }
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
 
             // ---- this partition's min / max (Eq. 7, Eq. 8): lanes sharing channels, then warps
 #pragma unroll
-            for (int j = 0; j < G::NWORD; ++j) {
+            for (int j = 0; j < G::NPW; ++j) {
 #pragma unroll
                 for (int o = G::LPR; o < 32; o <<= 1) {
                     mn[j] = G::E::min2(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
@@ -249,14 +249,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             }
             uint32_t* stats_t = stats + ((buf * 2 + tensor) * G::WT) * 2 * STAT_WORDS;
             if (rl == 0) {
-                uint32_t* st = stats_t + wj * 2 * STAT_WORDS;
-#pragma unroll
-                for (int v = 0; v < G::V; ++v)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        st[(v * G::LPR + cg) * 4 + c] = mn[v * 4 + c];
-                        st[STAT_WORDS + (v * G::LPR + cg) * 4 + c] = mx[v * 4 + c];
-                    }
+                store_stats_row<G>(stats_t + wj * 2 * STAT_WORDS, mn, mx, cg);
             }
             named_bar_sync(kBarTensor + tensor, WTE * 32);
             // sigma of this tensor is complete: hand the slot to the select warps
@@ -308,7 +301,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                         for (int j = etid; j < k; j += kWsSelThreads) P.idx_out[o + j] = row0 + kept[j];
                     } else if (P.K_out != nullptr && !sel_moves(i)) {
                         for (int j = etid; j < k; j += kWsSelThreads)
-                            *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::D) = row0 + kept[j];
+                            *reinterpret_cast<int32_t*>(P.K_out + (o + j) * G::ROW16) = row0 + kept[j];
                     }
                 }
                 // Long partitions: the select warps, idle most of the time, move the kept rows of
@@ -317,8 +310,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 // holding up the streamers; with short partitions they have no time to spare.
                 if (sel_moves(i) && P.K_out != nullptr)
                     emit_kept<kWsSelThreads, G::VPR, 16>(P.K, P.V, make_rowmap(P, u),
-                                                         P.K_out + (long long)u * P.L_R * G::D,
-                                                         P.V_out + (long long)u * P.L_R * G::D, sink + p * L,
+                                                         P.K_out + (long long)u * P.L_R * G::ROW16,
+                                                         P.V_out + (long long)u * P.L_R * G::ROW16, sink + p * L,
                                                          sink + p * k, kept, k, nullptr, etid);
                 __threadfence_block();  // the positions above are visible before the count below
                 sync_sel();             // every thread is done with kept[] and has written its share
@@ -420,7 +413,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 if (lane == 0) {
                     bulk_wait_read_all();
                     fence_proxy_async();
-                    mbar_arrive_expect_tx(copy_bar + 8 * st, uint32_t(2 * nr) * G::D * 2);
+                    mbar_arrive_expect_tx(copy_bar + 8 * st, uint32_t(2 * nr) * G::ROWB);
                 }
                 __syncwarp();
                 const uint32_t dK = stage_u32 + uint32_t(2 * st) * CHUNK_BYTES, dV = dK + CHUNK_BYTES;
@@ -435,22 +428,22 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 }
                 if (kind == 1 && contiguous) {
                     if (PAGED) {
-                        fetch_rows(P.K, um, src, nr, dK, copy_bar + 8 * st, G::D * 2, true, lane);
-                        fetch_rows(P.V, um, src, nr, dV, copy_bar + 8 * st, G::D * 2, true, lane);
+                        fetch_rows(P.K, um, src, nr, dK, copy_bar + 8 * st, G::ROWB, true, lane);
+                        fetch_rows(P.V, um, src, nr, dV, copy_bar + 8 * st, G::ROWB, true, lane);
                     } else if (lane == 0) {
-                        bulk_g2s(dK, P.K + um.base + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
-                        bulk_g2s(dV, P.V + um.base + (long long)src * P.ss, uint32_t(nr) * G::D * 2, copy_bar + 8 * st);
+                        bulk_g2s(dK, P.K + um.base + (long long)src * P.ss, uint32_t(nr) * G::ROWB, copy_bar + 8 * st);
+                        bulk_g2s(dV, P.V + um.base + (long long)src * P.ss, uint32_t(nr) * G::ROWB, copy_bar + 8 * st);
                     }
                 } else if (lane < nr) {  // one row of K and of V per lane
                     int row = src + lane;
                     if (kind == 2) {
                         __threadfence_block();
                         row = P.idx_out != nullptr ? __ldcg(P.idx_out + o + lane)
-                                                   : __ldcg(reinterpret_cast<const int32_t*>(P.K_out + (o + lane) * G::D));
+                                                   : __ldcg(reinterpret_cast<const int32_t*>(P.K_out + (o + lane) * G::ROW16));
                     }
                     const long long ro = um.off(row);
-                    bulk_g2s(dK + uint32_t(lane) * G::D * 2, P.K + ro, G::D * 2, copy_bar + 8 * st);
-                    bulk_g2s(dV + uint32_t(lane) * G::D * 2, P.V + ro, G::D * 2, copy_bar + 8 * st);
+                    bulk_g2s(dK + uint32_t(lane) * G::ROWB, P.K + ro, G::ROWB, copy_bar + 8 * st);
+                    bulk_g2s(dV + uint32_t(lane) * G::ROWB, P.V + ro, G::ROWB, copy_bar + 8 * st);
                 }
             }
             if (pending) {  // the chunk loaded before this one goes out
@@ -462,8 +455,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                 } else if (lane == 0) {
                     fence_proxy_async();
                     const uint32_t sK = stage_u32 + uint32_t(2 * pst) * CHUNK_BYTES, sV = sK + CHUNK_BYTES;
-                    bulk_s2g(P.K_out + po * G::D, sK, uint32_t(pnr) * G::D * 2);
-                    bulk_s2g(P.V_out + po * G::D, sV, uint32_t(pnr) * G::D * 2);
+                    bulk_s2g(P.K_out + po * G::ROW16, sK, uint32_t(pnr) * G::ROWB);
+                    bulk_s2g(P.V_out + po * G::ROW16, sV, uint32_t(pnr) * G::ROWB);
                     bulk_commit();
                 }
             }
@@ -509,8 +502,8 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
             RowMap um;  // PAGED only
             if (PAGED) um = make_rowmap(P, u);
             const long long o = (long long)u * P.L_R + sink + p * k;
-            uint16_t* dstK = P.K_out + o * G::D;
-            uint16_t* dstV = P.V_out + o * G::D;
+            uint16_t* dstK = P.K_out + o * G::ROW16;
+            uint16_t* dstV = P.V_out + o * G::ROW16;
             for (int g0 = warp; g0 < ngroups; g0 += NWALL * UG) {
                 int src[UG][IPL];
                 uint4 buf[UG][IPL];
@@ -523,7 +516,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                         if (g0 + q * NWALL < ngroups && j < k)
                             src[q][e] = P.idx_out != nullptr
                                             ? __ldcg(P.idx_out + o + j)
-                                            : __ldcg(reinterpret_cast<const int32_t*>(dstK + (long long)j * G::D));
+                                            : __ldcg(reinterpret_cast<const int32_t*>(dstK + (long long)j * G::ROW16));
                     }
                 __syncwarp();  // every parked position of this pass is read before a row is overwritten
 #pragma unroll
@@ -544,7 +537,7 @@ __global__ void __launch_bounds__(G::NT + kWsEpiWarps * 32, 1) lagkv_ws_kernel(c
                             const int va = (e * 32 + lane) % RV;
                             const int j = (g0 + q * NWALL) * GR + (e * 32 + lane) / RV;
                             uint16_t* dp = va >= G::VPR ? dstV : dstK;
-                            st_stream(reinterpret_cast<uint4*>(dp + (long long)j * G::D) + (va % G::VPR), buf[q][e]);
+                            st_stream(reinterpret_cast<uint4*>(dp + (long long)j * G::ROW16) + (va % G::VPR), buf[q][e]);
                         }
             }
         }

@@ -70,12 +70,21 @@ def make_kv(B: int, H: int, S: int, D: int, seed: int, sigma_k: float = 1.0, sig
         k[..., :half] = a * cos - b * sin
         k[..., half:] = b * cos + a * sin
         del a, b, cos, sin, ang
-    K = k.to(dtype)
+    K = _store(k, dtype)
     del k
     v = torch.randn((B, H, S, D), generator=g, device=dev, dtype=torch.float32)
     v *= torch.exp(sigma_v * torch.randn((B, H, S, 1), generator=g, device=dev, dtype=torch.float32))
-    V = v.to(dtype)
+    V = _store(v, dtype)
     return K, V
+
+
+def _store(x: torch.Tensor, dtype) -> torch.Tensor:
+    """Round fp32 draws to the cache's storage format.  fp8 (e4m3) holds at most 448: the draws are
+    first divided by a per-tensor scale (largest magnitude -> 400), which is what a quantising
+    engine does and what the compress pass never needs to know (it cancels in Eq. 9)."""
+    if dtype == torch.float8_e4m3fn:
+        return (x * (400.0 / float(x.abs().max()))).to(dtype)
+    return x.to(dtype)
 
 
 def make_workload_layer(w: Workload, layer: int, device="cpu", S: int | None = None):
@@ -85,7 +94,10 @@ def make_workload_layer(w: Workload, layer: int, device="cpu", S: int | None = N
 
 
 def to_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 (or fp16) tensor -> numpy uint16 array of the same shape (bit patterns, on the host)."""
+    """bf16 / fp16 tensor -> numpy uint16 array of the same shape, fp8 tensor -> uint8 array (bit
+    patterns, on the host)."""
+    if t.dtype == torch.float8_e4m3fn:
+        return t.detach().contiguous().view(torch.uint8).cpu().numpy()
     assert t.dtype in (torch.bfloat16, torch.float16)
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 

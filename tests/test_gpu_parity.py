@@ -35,6 +35,12 @@ def binding():
     return b
 
 
+def storage_of(oracle, dtype):
+    """The oracle's name for a torch storage format."""
+    return {torch.bfloat16: oracle.STORAGE_BF16, torch.float16: oracle.STORAGE_FP16,
+            torch.float8_e4m3fn: oracle.STORAGE_FP8_E4M3}[dtype]
+
+
 def check_against_oracle(oracle, Kb, Vb, sink, L, k, ddof, out, stats=None, variant=0, storage=0):
     """Compare a GPU prefill result ``out`` (numpy arrays) with the oracle on bit patterns."""
     ref = oracle.compress(Kb, Vb, sink, L, k, ddof=ddof, variant=variant, storage=storage)
@@ -81,7 +87,7 @@ def run_prefill(binding, oracle, B, H, D, S, sink, L, k, seed=0, ddof=1, tune=No
     host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
             "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
     return check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, ddof, host, variant=variant,
-                                storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
+                                storage=storage_of(oracle, dtype))
 
 
 # ------------------------------------------------------------------------------- prefill
@@ -242,7 +248,7 @@ def test_rows_only_warp_specialised_every_head_dim(binding, oracle, D, dtype):
     host = {"L_R": full["L_R"], "idx": full["idx"].cpu().numpy(), "K_out": synth.to_bits(full["K_out"]),
             "V_out": synth.to_bits(full["V_out"]), "scores": full["scores"].cpu().numpy()}
     check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host,
-                         storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
+                         storage=storage_of(oracle, dtype))
     L_R = full["L_R"]
     for run in range(6):
         out = {"K_out": torch.full((B, H, L_R, D), -3.0, dtype=dtype, device="cuda:0"),
@@ -353,7 +359,7 @@ def run_l2norm(binding, oracle, B, H, D, S, sink, L, k, seed, tune=None, dtype=t
     assert plan.read_status(ws)[0] == 0
     Kb, Vb = synth.to_bits(K), synth.to_bits(V)
     ref = oracle.compress(Kb, Vb, sink, L, k, variant=oracle.VARIANT_L2NORM,
-                          storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
+                          storage=storage_of(oracle, dtype))
     idx = out["idx"].cpu().numpy()
     n_c = ref["n_c"]
     assert out["L_R"] == ref["L_R"]
@@ -537,7 +543,7 @@ def test_paged_prefill(binding, oracle, D, L, k, page, pad, dtype, variant):
     assert plan.read_status(ws)[0] == 0
     host = {"L_R": out["L_R"], "idx": out["idx"].cpu().numpy(), "K_out": synth.to_bits(out["K_out"]),
             "V_out": synth.to_bits(out["V_out"]), "scores": out["scores"].cpu().numpy()}
-    storage = oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16
+    storage = storage_of(oracle, dtype)
     if variant == 2:      # Eq. 16: relative tolerance on the norms; same picks as the contiguous call
         flat = binding.Plan(B, H, D, sink, L, keep_k=k, variant=variant, device=0, dtype=dtype)
         ref = flat.compress_prefill(K, V, ws, want_scores=True)
@@ -656,7 +662,7 @@ def append_case(binding, oracle, B, H, D, S_cap, sink, L, k, seq, stat, max_chun
     st = plan.read_status(ws)
     Kr, Vr, seq_r, stat_r, kept = oracle.compress_append(
         Kb, Vb, np.array(seq), np.array(stat), L, k, variant=variant,
-        storage=oracle.STORAGE_FP16 if dtype == torch.float16 else oracle.STORAGE_BF16)
+        storage=storage_of(oracle, dtype))
     return dict(K=synth.to_bits(K), V=synth.to_bits(V), seq=seq_d.cpu().numpy(), stat=stat_d.cpu().numpy(),
                 idx=None if idx_out is None else idx_out.cpu().numpy(), status=st,
                 Kr=Kr, Vr=Vr, seq_r=seq_r, stat_r=stat_r, kept=kept, K0=Kb, V0=Vb)
@@ -1236,3 +1242,80 @@ def test_c_program_prefill_parity(binding, tmp_path):
                     f"-L{cuda / 'lib64'}", "-lcudart", f"-Wl,-rpath,{cuda / 'lib64'}", "-lm"], check=True)
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0 and out.stdout.startswith("ok"), out.stdout + out.stderr
+
+
+# ------------------------------------------------------------------------------- fp8 caches
+FP8 = torch.float8_e4m3fn
+
+
+@pytest.mark.parametrize("L,k,S_extra,tune,variant", [
+    (64, 16, 60, None, 0), (100, 25, 7, None, 0), (128, 16, 100, dict(warps=100, tile_rows=32, stages=2, ctas_per_sm=1), 0),
+    (128, 32, 0, dict(warps=100, tile_rows=16, stages=2, ctas_per_sm=1), 0), (256, 64, 255, None, 0), (512, 128, 3, dict(warps=12, tile_rows=16), 0),
+    (1024, 256, 1008, None, 0), (2048, 256, 100, dict(warps=8, tile_rows=32, stages=3, ctas_per_sm=1), 0),
+    (256, 1, 17, dict(warps=4, tile_rows=32, stages=3, ctas_per_sm=2), 0), (37, 5, 36, None, 0),
+    (128, 32, 11, None, 1), (512, 128, 100, None, 1), (300, 75, 7, None, 2)])
+def test_fp8_prefill(binding, oracle, L, k, S_extra, tune, variant):
+    """fp8 (e4m3) caches through every kernel family and scoring variant: scores within the fp32
+    bars of the oracle's reading of the same bytes, picks exact or explained, rows byte for byte."""
+    n = 5 if L >= 512 else 9
+    if variant == 2:
+        run_l2norm(binding, oracle, 2, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + 3, tune=tune, dtype=FP8)
+    else:
+        run_prefill(binding, oracle, 2, 3, 128, 4 + n * L + S_extra, 4, L, k, seed=L + k, tune=tune, variant=variant,
+                    dtype=FP8)
+
+
+def test_fp8_many_units_rows_only_and_paged(binding, oracle):
+    """fp8 on the warp-specialised kernel with several slots per CTA: the run without indices (parked
+    positions) and the run on a paged copy of the cache give the same bytes as the checked run."""
+    B, H, D, sink, L, k = 8, 5, 128, 16, 256, 64
+    S = sink + 21 * L + 77
+    K, V = synth.make_kv(B, H, S, D, seed=88, device="cuda:0", dtype=FP8)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0, dtype=FP8)
+    assert plan.launch_info(S)["kernel"] == "lagkv_ws_kernel"
+    ws = plan.new_workspace()
+    full = plan.compress_prefill(K, V, ws, want_scores=True)
+    host = {"L_R": full["L_R"], "idx": full["idx"].cpu().numpy(), "K_out": synth.to_bits(full["K_out"]),
+            "V_out": synth.to_bits(full["V_out"]), "scores": full["scores"].cpu().numpy()}
+    check_against_oracle(oracle, synth.to_bits(K), synth.to_bits(V), sink, L, k, 1, host,
+                         storage=oracle.STORAGE_FP8_E4M3)
+    u8 = lambda t: t.view(torch.uint8)
+    rows = plan.compress_prefill(K, V, ws, want_idx=False)
+    assert torch.equal(u8(rows["K_out"]), u8(full["K_out"])) and torch.equal(u8(rows["V_out"]), u8(full["V_out"]))
+    Kp, Vp, table = paginate(u8(K), u8(V), 64, seed=3)
+    paged = plan.compress_prefill_paged(Kp.view(FP8), Vp.view(FP8), table, S, ws, want_scores=True)
+    assert plan.read_status(ws)[0] == 0
+    assert torch.equal(paged["idx"], full["idx"]) and torch.equal(paged["scores"], full["scores"])
+    assert torch.equal(u8(paged["K_out"]), u8(full["K_out"])) and torch.equal(u8(paged["V_out"]), u8(full["V_out"]))
+
+
+@pytest.mark.parametrize("L,k,chunks,tune", [(64, 16, 3, None), (512, 128, 1, dict(warps=CLUSTER, tile_rows=2, stages=2, ctas_per_sm=2)),
+                                             (512, 128, 1, dict(warps=4, tile_rows=32, stages=3, ctas_per_sm=2)),
+                                             (96, 24, 1, dict(warps=CLUSTER, tile_rows=1, stages=2, ctas_per_sm=2))])
+def test_fp8_append(binding, oracle, L, k, chunks, tune):
+    sink = 8
+    stat = [sink, sink + 2 * k, sink]
+    seq = [stat[0] + (chunks + 1) * L + 3, stat[1] + (chunks + 1) * L, stat[2] + 2 * L - 1]
+    r = append_case(binding, oracle, 3, 2, 128, max(seq) + 9, sink, L, k, seq, stat, chunks, seed=L + chunks, tune=tune,
+                    dtype=FP8)
+    check_append(r, 3)
+
+
+def test_fp8_scores_do_not_depend_on_the_quantisation_scale(binding):
+    """A power-of-two rescale of a whole fp8 cache (what a different per-tensor scale of the
+    caller's quantiser amounts to) leaves scores and picks bit-identical: Eq. 9 cancels it."""
+    B, H, D, sink, L, k = 2, 2, 128, 4, 128, 32
+    S = sink + 6 * L + 9
+    K, V = synth.make_kv(B, H, S, D, seed=5, device="cuda:0")                 # bf16 draws
+    scale = 8.0 / float(K.float().abs().max())
+    K8a, V8a = (K.float() * scale).to(FP8), (V.float() * scale).to(FP8)
+    for t in (K8a, V8a):      # flush what would be subnormal (a rescale of those is not exact)
+        t.view(torch.uint8)[(t.view(torch.uint8) & 0x78) == 0] = 0
+    big = lambda t: (t.float() * 16.0).to(FP8)                                # exact: exponent + 4, far from both ends
+    K8b, V8b = big(K8a), big(V8a)
+    assert torch.equal(K8b.float(), K8a.float() * 16.0)
+    plan = binding.Plan(B, H, D, sink, L, keep_k=k, device=0, dtype=FP8)
+    ws = plan.new_workspace()
+    a = plan.compress_prefill(K8a, V8a, ws, want_scores=True)
+    b = plan.compress_prefill(K8b, V8b, ws, want_scores=True)
+    assert torch.equal(a["scores"], b["scores"]) and torch.equal(a["idx"], b["idx"])

@@ -33,6 +33,11 @@ MUTANTS = {
     "fp16_exponent_bias": ("ldexp(1.0 + (double)frac / 1024.0, e - 15);", "ldexp(1.0 + (double)frac / 1024.0, e - 16);"),
     "fp16_subnormal_scale": ("ldexp((double)frac, -24);", "ldexp((double)frac, -25);"),
     "fp16_fraction_width": ("(double)frac / 1024.0", "(double)frac / 2048.0"),
+    "fp8_exponent_bias": ("ldexp(1.0 + (double)frac / 8.0, e - 7);", "ldexp(1.0 + (double)frac / 8.0, e - 8);"),
+    "fp8_subnormal_scale": ("ldexp((double)frac, -9);", "ldexp((double)frac, -10);"),
+    "fp8_fraction_width": ("(double)frac / 8.0", "(double)frac / 16.0"),
+    "fp8_has_infinities": ("else if (e == 15 && frac == 7)\n        v = NAN;", "else if (e == 15)\n        v = frac ? NAN : INFINITY;"),
+    "fp8_flag_ignored": ("if (storage == LAGKV_ORACLE_FP8_E4M3) return fp8_e4m3_to_double(bits);", ""),
     "storage_flag_ignored": ("return storage == LAGKV_ORACLE_FP16 ? fp16_to_double(bits) : bf16_to_double(bits);",
                              "return bf16_to_double(bits);"),
 }
@@ -65,6 +70,8 @@ def run_pins(mod, only=None):
         ("decode", lambda: pins.test_decode_every_bit_pattern(mod)),
         ("fp16_same_values", lambda: pins.test_fp16_storage_same_values_same_result(mod, 1)),
         ("fp16_only", lambda: pins.test_fp16_storage_values_only_fp16_holds(mod)),
+        ("fp8_decode", lambda: pins.test_decode_fp8_every_byte(mod)),
+        ("fp8_same_values", lambda: pins.test_fp8_storage_same_values_same_result(mod, 1)),
     ]
     failed = []
     for name, fn in checks:

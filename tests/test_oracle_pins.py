@@ -104,6 +104,48 @@ def test_fp16_storage_values_only_fp16_holds(oracle):
     assert not np.allclose(wrong, want, rtol=1e-3)
 
 
+def test_decode_fp8_every_byte(oracle):
+    """The oracle's reading of all 256 fp8 (e4m3, finite-only) bytes against torch's conversion of
+    the same bytes and against the format's definition: (-1)^s 2^(e-7) (1 + m/8), subnormals
+    m/8 x 2^-6, no infinities, 0x7f and 0xff the only NaNs."""
+    import torch
+    allbytes = np.arange(256, dtype=np.uint8)
+    got = oracle.decode(allbytes, oracle.STORAGE_FP8_E4M3)
+    want = torch.from_numpy(allbytes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.isnan(got).sum() == 2 and np.isnan(got[0x7f]) and np.isnan(got[0xff])
+    ok = ~np.isnan(want)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.array_equal(got[ok], want[ok]) and np.array_equal(np.signbit(got[ok]), np.signbit(want[ok]))
+    for byte, value in ((0x00, 0.0), (0x38, 1.0), (0x3c, 1.5), (0x40, 2.0), (0x7e, 448.0), (0x01, 2.0 ** -9),
+                        (0x07, 7 * 2.0 ** -9), (0x08, 2.0 ** -6), (0xc0, -2.0), (0xfe, -448.0)):
+        assert got[byte] == value, (hex(byte), got[byte], value)
+    s, e, m = allbytes >> 7, (allbytes >> 3) & 15, allbytes & 7
+    formula = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7)) * np.where(s == 1, -1.0, 1.0)
+    assert np.array_equal(got[ok], formula[ok])
+
+
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_fp8_storage_same_values_same_result(oracle, ddof):
+    """Values that bf16 and fp8 both hold exactly (small integers and halves) give the same scores
+    and picks whichever format stores them; the kept rows come back as the stored bytes."""
+    import torch
+    rng = np.random.default_rng(21 + ddof)
+    S, L, D, k, n = 3, 8, 4, 3, 4
+    Ls = S + n * L + 5
+    Kf = rng.integers(-16, 17, (1, 1, Ls, D)) / 2.0      # multiples of 1/2 up to 8: at most 4 significant bits
+    Vf = rng.integers(-16, 17, (1, 1, Ls, D)) / 2.0
+    K8 = torch.from_numpy(Kf).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    V8 = torch.from_numpy(Vf).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(oracle.decode(K8, oracle.STORAGE_FP8_E4M3), Kf)
+    a = oracle.compress(bits(Kf), bits(Vf), S, L, k, ddof=ddof)
+    b = oracle.compress(K8, V8, S, L, k, ddof=ddof, storage=oracle.STORAGE_FP8_E4M3)
+    assert np.array_equal(a["idx"], b["idx"]) and np.array_equal(a["scores"], b["scores"])
+    assert b["K_out"].dtype == np.uint8
+    assert np.array_equal(b["K_out"], np.take_along_axis(K8, b["idx"][..., None].astype(np.int64), axis=2))
+    assert np.array_equal(b["V_out"], np.take_along_axis(V8, b["idx"][..., None].astype(np.int64), axis=2))
+    assert brute.compress_head(Kf[0, 0].tolist(), Vf[0, 0].tolist(), S, L, k, ddof) == b["idx"][0, 0].tolist()
+
+
 # ------------------------------------------------------------------ worked examples
 @pytest.mark.parametrize("name", ["hand_case_1.txt", "hand_case_2.txt"])
 @pytest.mark.parametrize("ddof", [0, 1])
