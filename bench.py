@@ -2,7 +2,7 @@
 """Benchmark of the LagKV compress pass on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
-                    [--variant lagkv|localkv|l2norm] [--storage bf16|fp16] [--layers N] [--tune w,t,s,c]
+                    [--variant lagkv|localkv|l2norm] [--storage bf16|fp16|fp8] [--layers N] [--tune w,t,s,c]
                     [--paged PAGE_ROWS]
     python bench.py --workload sweep --sweep [--sweep-B 1,8]   # one JSON line per (L, r, B) cell of the sweep
     python bench.py --workload decode_append --append          # the incremental pass, one triggering call per step
@@ -55,11 +55,11 @@ SWEEP_R = (0.5, 0.25, 0.125, 0.0625)
 TRAFFIC_JSON = ROOT / "profiles" / "ncu_traffic.json"
 
 
-def algorithmic_bytes(w, L_R: int, variant: int = 0) -> int:
+def algorithmic_bytes(w, L_R: int, variant: int = 0, elem_bytes: int = 2) -> int:
     """Every input row read once, every output row written once, index list written once.
     The L2-norm variant scores from K alone: of V only the L_R output rows are read."""
     units = w.layers * w.B * w.H
-    row = w.D * 2
+    row = w.D * elem_bytes
     if variant == 2:
         return units * (w.S * row + L_R * row + L_R * 2 * row + 4 * L_R)
     return units * ((w.S + L_R) * 2 * row + 4 * L_R)
@@ -517,7 +517,7 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
     """One workload on this rank; returns the JSON line (rank 0) or None."""
     import torch.distributed as dist
     Bf = w.layers * w.B
-    store = torch.float16 if args.storage == "fp16" else torch.bfloat16
+    store = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp8": torch.float8_e4m3fn}[args.storage]
     K = torch.empty((Bf, w.H, w.S, w.D), dtype=store, device=dev)
     V = torch.empty_like(K)
     for layer in range(w.layers):
@@ -572,7 +572,7 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
         dist.barrier()
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream(dev)
-    input_bytes = 2 * K.numel() * 2
+    input_bytes = 2 * K.numel() * K.element_size()
     flush_l2 = input_bytes < 4 * 126e6          # small caches would be served from the 126 MB L2
     wall0 = time.time()
     ms_total = time_prefill(torch, step, args.steps, stream, flush_l2, dev)
@@ -647,7 +647,7 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
     if rank != 0:
         return None
     peak, peak_src = measured_peak()
-    alg = algorithmic_bytes(w, L_R, variant)
+    alg = algorithmic_bytes(w, L_R, variant, 1 if args.storage == "fp8" else 2)
     achieved = alg / (ms_step * 1e-3) / 1e9
     captured = not args.layers and not args.tune and variant == 0 and args.storage == "bf16" and not args.paged
     traffic = captured_traffic(w.name) if captured else None   # counters of exactly this launch, else null
@@ -733,8 +733,8 @@ def main():
     ap.add_argument("--tune", default="", help="warps,tile_rows,stages,ctas_per_sm override")
     ap.add_argument("--variant", default="lagkv", choices=["lagkv", "localkv", "l2norm"],
                     help="scoring variant of Section 4.3 (the headline metric is lagkv)")
-    ap.add_argument("--storage", default="bf16", choices=["bf16", "fp16"],
-                    help="storage format of the caches (fp16: device-timed pass only)")
+    ap.add_argument("--storage", default="bf16", choices=["bf16", "fp16", "fp8"],
+                    help="storage format of the caches (fp16, fp8 = e4m3: device-timed pass only)")
     ap.add_argument("--append", action="store_true",
                     help="time the incremental pass instead: every step is one lagkv_compress_append call in which "
                          "every sequence has just completed a partition and its lag partition (single GPU)")
