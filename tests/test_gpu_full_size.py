@@ -3,7 +3,8 @@
 size over the whole result, and EVERY partition's scores and kept indices against the float64
 oracle, which replays the workload layer by layer (cell by cell for the sweep).  The counters
 (largest score error, partitions whose index set differs, near-ties under both thresholds) are
-printed and written to ``gpurun_out/parity_counters.json`` when that folder exists."""
+printed and, when the environment names a folder in ``LAGKV_COUNTERS_DIR``, written to
+``parity_counters.json`` there."""
 import json
 import os
 
@@ -48,8 +49,8 @@ def oracle_all_partitions(oracle, K, V, out, sink, L, k, units_per_step):
 
 def record_counters(name, counters):
     print(f"{name}: {json.dumps(counters)}")
-    root = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(root):
+    root = os.environ.get("LAGKV_COUNTERS_DIR", "")
+    if root and os.path.isdir(root):
         path = os.path.join(root, "parity_counters.json")
         allc = json.load(open(path)) if os.path.exists(path) else {}
         allc[name] = counters
