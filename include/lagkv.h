@@ -309,6 +309,11 @@ int lagkv_gather(lagkv_plan_t plan, const void *K, const void *V, int64_t S_in,
                  const int32_t *idx, int64_t n_idx, void *K_out, void *V_out, void *workspace,
                  void *cuda_stream);
 
+/* lagkv_gather() reading a paged cache (see lagkv_paged_layout); outputs contiguous as there. */
+int lagkv_gather_paged(lagkv_plan_t plan, const void *K_pool, const void *V_pool, const lagkv_paged_layout *layout,
+                       int64_t S_in, const int32_t *idx, int64_t n_idx, void *K_out, void *V_out, void *workspace,
+                       void *cuda_stream);
+
 /*
  * Synchronise cuda_stream, copy the status block to the host and clear it.  workspace == NULL
  * names the status block of the library's built-in scratch on the plan's device (the one

@@ -30,7 +30,7 @@ EXPORTS = (
     "lagkv_keep_for_target", "lagkv_lengths_after", "lagkv_workspace_bytes", "lagkv_workspace_init",
     "lagkv_compress_prefill", "lagkv_compress_prefill_host", "lagkv_host_staging_bytes",
     "lagkv_compress_append", "lagkv_compress_append_noalloc", "lagkv_compress_prefill_paged",
-    "lagkv_compress_append_paged", "lagkv_gather",
+    "lagkv_compress_append_paged", "lagkv_gather", "lagkv_gather_paged",
     "lagkv_read_status",
     "lagkv_launch_info", "lagkv_plan_tune", "lagkv_selftest_bounded_wait", "lagkv_status_string", "lagkv_version",
 )
@@ -106,6 +106,8 @@ def load_library() -> ctypes.CDLL:
     lib.lagkv_compress_append_paged.restype = ctypes.c_int
     lib.lagkv_compress_append_paged.argtypes = [vp, vp, vp, ctypes.POINTER(lagkv_paged_layout), vp, vp, i32, vp, vp, vp,
                                                 sz, vp]
+    lib.lagkv_gather_paged.restype = ctypes.c_int
+    lib.lagkv_gather_paged.argtypes = [vp, vp, vp, ctypes.POINTER(lagkv_paged_layout), i64, vp, i64, vp, vp, vp, vp]
     lib.lagkv_gather.restype = ctypes.c_int
     lib.lagkv_gather.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
     lib.lagkv_read_status.restype = ctypes.c_int
@@ -341,6 +343,19 @@ class Plan:
             int(max_new_chunks), _ptr(idx_out), _ptr(scores_out), _ptr(workspace), workspace.numel(),
             _stream(self._dev()))
         _check(rc, "lagkv_compress_append_paged")
+
+    def gather_paged(self, K_pool, V_pool, block_table, idx, S_in, workspace=None, strides=None):
+        """``lagkv_gather_paged``: rows ``idx`` ``[B, H, n_idx]`` of a paged cache."""
+        self._check_cache(K_pool, "K_pool")
+        lay = self._paged(K_pool, block_table, strides)
+        c, dev = self.cfg, self._dev()
+        n_idx = int(idx.shape[-1])
+        K_out = torch.empty((c.B, c.H_kv, n_idx, c.D), dtype=self.dtype, device=dev)
+        V_out = None if V_pool is None else torch.empty_like(K_out)
+        rc = self.lib.lagkv_gather_paged(self.handle, _ptr(K_pool), _ptr(V_pool), ctypes.byref(lay), int(S_in), _ptr(idx),
+                                         n_idx, _ptr(K_out), _ptr(V_out), _ptr(workspace), _stream(dev))
+        _check(rc, "lagkv_gather_paged")
+        return K_out, V_out
 
     def gather(self, K, V, idx, workspace=None, S_in=None):
         """``lagkv_gather``: rows ``idx`` ``[B, H, n_idx]`` int32 of K (and V, may be None)."""

@@ -805,8 +805,9 @@ int lagkv_compress_append_paged(lagkv_plan_t plan, void* K_pool, void* V_pool, c
                        workspace, workspace_bytes, cuda_stream, layout);
 }
 
-int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, const int32_t* idx, int64_t n_idx,
-                 void* K_out, void* V_out, void* workspace, void* cuda_stream) {
+static int gather_impl(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, const int32_t* idx,
+                       int64_t n_idx, void* K_out, void* V_out, void* workspace, void* cuda_stream,
+                       const lagkv_paged_layout* paged) {
     if (plan == nullptr || K == nullptr || K_out == nullptr || idx == nullptr || plan->cfg.device < 0)
         return LAGKV_EINVAL;
     if ((V == nullptr) != (V_out == nullptr)) return LAGKV_EINVAL;
@@ -816,7 +817,11 @@ int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, 
         return LAGKV_EINVAL;
     const lagkv_config& c = plan->cfg;
     Strides st;
-    if (resolve_strides(c, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    if (paged != nullptr) {
+        if (resolve_paged(c, paged, S_in, &st) != LAGKV_OK) return LAGKV_EINVAL;
+    } else if (resolve_strides(c, S_in, &st) != LAGKV_OK) {
+        return LAGKV_EINVAL;
+    }
     if (n_idx == 0) return LAGKV_OK;
     DeviceGuard guard(c.device);
     const long long U = (long long)c.B * c.H_kv;
@@ -830,6 +835,18 @@ int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, 
         vpr, idx, n_idx, static_cast<uint16_t*>(K_out), static_cast<uint16_t*>(V_out), U,
         static_cast<int32_t*>(workspace));
     return check_launch();
+}
+
+int lagkv_gather(lagkv_plan_t plan, const void* K, const void* V, int64_t S_in, const int32_t* idx, int64_t n_idx,
+                 void* K_out, void* V_out, void* workspace, void* cuda_stream) {
+    return gather_impl(plan, K, V, S_in, idx, n_idx, K_out, V_out, workspace, cuda_stream, nullptr);
+}
+
+int lagkv_gather_paged(lagkv_plan_t plan, const void* K_pool, const void* V_pool, const lagkv_paged_layout* layout,
+                       int64_t S_in, const int32_t* idx, int64_t n_idx, void* K_out, void* V_out, void* workspace,
+                       void* cuda_stream) {
+    if (layout == nullptr) return LAGKV_EINVAL;
+    return gather_impl(plan, K_pool, V_pool, S_in, idx, n_idx, K_out, V_out, workspace, cuda_stream, layout);
 }
 
 int lagkv_read_status(lagkv_plan_t plan, void* workspace, void* cuda_stream, int32_t host_status[4]) {

@@ -585,6 +585,18 @@ def test_paged_prefill_warp_specialised_many_units(binding, page, dtype):
     assert torch.equal(Ko, ref["K_out"]) and torch.equal(Vo, ref["V_out"])
 
 
+def test_paged_gather(binding, oracle):
+    B, H, D, S, page = 2, 3, 128, 300, 32
+    K, V = synth.make_kv(B, H, S, D, seed=44, device="cuda:0")
+    Kp, Vp, table = paginate(K, V, page, seed=2)
+    g = torch.Generator(device="cuda:0").manual_seed(1)
+    idx = torch.randint(0, S, (B, H, 77), generator=g, device="cuda:0", dtype=torch.int32)
+    plan = binding.Plan(B, H, D, 4, 64, keep_k=16, device=0)
+    Ko, Vo = plan.gather_paged(Kp, Vp, table, idx, S)
+    np.testing.assert_array_equal(synth.to_bits(Ko), oracle.gather(synth.to_bits(K), idx.cpu().numpy()))
+    np.testing.assert_array_equal(synth.to_bits(Vo), oracle.gather(synth.to_bits(V), idx.cpu().numpy()))
+
+
 def test_paged_prefill_identity_and_errors(binding, oracle):
     B, H, D, sink, L, k, page = 2, 2, 128, 8, 64, 16, 16
     S = sink + 2 * L - 1                                     # too short: identity
