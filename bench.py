@@ -199,7 +199,7 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    per_step = max(1.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    per_step = args.cpu_seconds or max(1.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
     layers_bits = host_layers(w, 2)
     vals = []
     last = None
@@ -688,9 +688,9 @@ def run_prefill(args, w, torch, binding, synth, shard, rank, world, local, dev, 
         layers_bits = [(synth.to_bits(K[l * w.B:(l + 1) * w.B]), synth.to_bits(V[l * w.B:(l + 1) * w.B]))
                        for l in range(min(4, w.layers))]
         del K, V
-        cb = time_oracle(w, layers_bits)
+        cb = time_oracle(w, layers_bits, seconds_target=args.cpu_seconds or 12.0)
         cb.pop("seconds"), cb.pop("tokens_heads")
-        one = time_oracle(w, layers_bits[:1], seconds_target=4.0, threads=1)
+        one = time_oracle(w, layers_bits[:1], seconds_target=(args.cpu_seconds or 12.0) / 3, threads=1)
         cb["single_thread_value"] = one["value"]
         line["cpu_baseline"] = cb
     return line
@@ -745,6 +745,9 @@ def main():
     ap.add_argument("--sweep-B", default="1,8", help="batch sizes of the sweep")
     ap.add_argument("--paged", type=int, default=0, help="read the cache through a block table with pages of N rows")
     ap.add_argument("--sustained", type=float, default=2.0, help="seconds of the sustained run (0 = skip)")
+    ap.add_argument("--cpu-seconds", type=float, default=0.0,
+                    help="CPU time of the oracle sample (default: 12 s in the cpu_baseline leg, up to 20 s per step "
+                         "of the reference arm)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
