@@ -208,6 +208,9 @@ int lagkv_compress_prefill_host(lagkv_plan_t plan, const void *K_host, const voi
  *               kept by this call (entries of skipped sequences are not written).
  *   scores_out  [B, H, max_new_chunks*L] fp32 or NULL.
  * The workspace must have been sized with the same max_new_chunks.
+ * With max_new_chunks == 1 (decode: at most one partition completes per call) and at most
+ * sm_count (b, h) units the launch is a grid of thread-block clusters, one cluster per unit,
+ * which keeps the window in shared memory between its two uses; it is still one launch.
  */
 int lagkv_compress_append(lagkv_plan_t plan, void *K_cache, void *V_cache, int64_t S_cap,
                           int32_t *seq_len, int32_t *static_len, int32_t max_new_chunks,
@@ -230,7 +233,8 @@ typedef struct {
     int32_t page_size;          /* rows per page: a power of two, >= 16                        */
     int64_t stride_page;        /* elements between pages          (0 = H_kv*stride_h)         */
     int64_t stride_h;           /* elements between heads in a page (0 = page_size*stride_s)   */
-    int64_t stride_s;           /* elements between rows in a page  (0 = D); multiples of 8    */
+    int64_t stride_s;           /* elements between rows in a page  (0 = D); all three strides
+                                   multiples of 16 bytes                                       */
 } lagkv_paged_layout;
 
 /*
