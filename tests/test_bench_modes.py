@@ -26,6 +26,21 @@ def test_algorithmic_bytes_and_traffic_record():
     assert bench.captured_traffic("no such workload") is None
 
 
+def test_gpus_flag_starts_its_own_ranks(monkeypatch):
+    """``--gpus N`` outside a torchrun environment re-launches the benchmark under
+    ``torch.distributed.run`` with N local ranks on 127.0.0.1 and the same arguments."""
+    sys.path.insert(0, ROOT)
+    import bench
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "7"])
+    assert bench.respawn_under_torchrun(4) == 0
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "4", "--steps", "7"]
+    assert os.path.basename(cmd[cmd.index("--master-port") + 2]) == "bench.py"
+
+
 def run_bench(*args):
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True,
                          timeout=600)
