@@ -79,7 +79,7 @@ enum lagkv_dtype {
                              per-head or per-channel scale the caller's quantiser uses, it
                              cancels in Eq. 9 (the same scale multiplies value, min and max),
                              so the scores are those of the stored bytes and the kept rows
-                             are copied byte for byte.  head_dim 128 only.                 */
+                             are copied byte for byte.                                     */
 };
 
 typedef struct {

@@ -18,7 +18,7 @@ namespace {
 
 // every compiled kernel: the three tables live in translation units of their own
 struct KernelTable {
-    static constexpr int kMaxEntries = 256;
+    static constexpr int kMaxEntries = 384;
     const KernelEntry* e[kMaxEntries];
     int n = 0;
     KernelTable() {
@@ -42,6 +42,8 @@ struct KernelTable {
         c = ws_paged_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
         c = fp8_kernels(&t);
+        for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
+        c = fp8_dims_kernels(&t);
         for (int i = 0; i < c && n < kMaxEntries; ++i) e[n++] = t + i;
     }
 };

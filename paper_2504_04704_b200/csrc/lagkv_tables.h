@@ -70,5 +70,6 @@ constexpr int kAppendPairTileRows = 16;
       &lagkv_ws_kernel<Geo<D, V, NWS, TR, DT>, 0, true>, &ws_smem_total_bytes<Geo<D, V, NWS, TR, DT>>, true }
 int ws_paged_kernels(const KernelEntry** table);      // lagkv_ws_kernel reading paged caches
 int fp8_kernels(const KernelEntry** table);           // every family for fp8 (e4m3) caches, head_dim 128
+int fp8_dims_kernels(const KernelEntry** table);      // ... head_dim 64, 96, 256
 
 }  // namespace lagkv

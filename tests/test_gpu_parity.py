@@ -1331,3 +1331,23 @@ def test_fp8_scores_do_not_depend_on_the_quantisation_scale(binding):
     a = plan.compress_prefill(K8a, V8a, ws, want_scores=True)
     b = plan.compress_prefill(K8b, V8b, ws, want_scores=True)
     assert torch.equal(a["scores"], b["scores"]) and torch.equal(a["idx"], b["idx"])
+
+
+@pytest.mark.parametrize("D", [64, 96, 256])
+@pytest.mark.parametrize("L,k,tune", [(64, 16, None), (128, 16, dict(warps=100, tile_rows=32, stages=2, ctas_per_sm=1)),
+                                      (256, 64, None), (1024, 256, None)])
+def test_fp8_head_dims(binding, oracle, D, L, k, tune):
+    """fp8 rows of 64, 96 and 256 bytes on the uniform, pair and (where compiled) warp-specialised kernels."""
+    n = 4 if L >= 512 else 7
+    run_prefill(binding, oracle, 2, 3, D, 16 + n * L + 37, 16, L, k, seed=D + L, tune=tune, dtype=FP8)
+
+
+@pytest.mark.parametrize("D", [64, 96, 256])
+def test_fp8_append_head_dims(binding, oracle, D):
+    """fp8 appends at the other head dims: several partitions (uniform kernel) and one (cluster)."""
+    sink, L, k = 8, 128, 32
+    for chunks in (2, 1):
+        stat = [sink, sink + k]
+        seq = [stat[0] + (chunks + 1) * L + 5, stat[1] + (chunks + 1) * L]
+        r = append_case(binding, oracle, 2, 2, D, max(seq) + 9, sink, L, k, seq, stat, chunks, seed=D + chunks, dtype=FP8)
+        check_append(r, 2)
